@@ -1,0 +1,190 @@
+"""TEST INFRASTRUCTURE -- ctypes loader for the fp64 CPU checker in kvmo.cpp.
+
+Only tests, the smoke check and the benchmark's CPU-baseline leg may import
+this module.  It never touches the CUDA library.
+"""
+from __future__ import annotations
+
+import ctypes
+import math
+import os
+import subprocess
+from dataclasses import dataclass
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "kvmo.cpp")
+_LIB = os.path.join(_HERE, "libkvmo.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile kvmo.cpp into libkvmo.so next to it (g++ with OpenMP)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.check_call(["g++", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c++17", "-o", tmp, _SRC])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.kvmo_num_threads.restype = ctypes.c_int
+    return _lib
+
+
+def num_threads() -> int:
+    return int(lib().kvmo_num_threads())
+
+
+def _p(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _f32(x) -> np.ndarray:
+    """Storage-dtype tensor/array -> contiguous fp32 numpy array (exact for bf16 and fp32)."""
+    if hasattr(x, "detach"):
+        x = x.detach().cpu().float().numpy()
+    return np.ascontiguousarray(x, dtype=np.float32)
+
+
+def sizes(S: int, budget: float, recent: float, heavy: float):
+    C, nr, nh = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
+    lib().kvmo_sizes(ctypes.c_int32(S), ctypes.c_double(budget), ctypes.c_double(recent), ctypes.c_double(heavy),
+                     ctypes.byref(C), ctypes.byref(nr), ctypes.byref(nh))
+    return C.value, nr.value, nh.value
+
+
+def scores(Q, K, scale: Optional[float] = None, want_lse: bool = False):
+    Q, K = _f32(Q), _f32(K)
+    B, Hq, S, D = Q.shape
+    Hkv = K.shape[1]
+    if scale is None:
+        scale = 1.0 / math.sqrt(D)
+    a = np.empty((B, Hkv, S), dtype=np.float64)
+    lse = np.empty((B, Hq, S), dtype=np.float64) if want_lse else None
+    lib().kvmo_scores(ctypes.c_int32(B), ctypes.c_int32(Hq), ctypes.c_int32(Hkv), ctypes.c_int32(S),
+                      ctypes.c_int32(D), ctypes.c_double(scale), _p(Q), _p(K), _p(a), _p(lse))
+    return (a, lse) if want_lse else a
+
+
+def keep(scores_: np.ndarray, n_r: int, n_h: int) -> np.ndarray:
+    a = np.ascontiguousarray(scores_, dtype=np.float64)
+    S = a.shape[-1]
+    U = a.size // S
+    out = np.empty(a.shape, dtype=np.uint8)
+    lib().kvmo_keep(ctypes.c_int64(U), ctypes.c_int32(S), ctypes.c_int32(n_r), ctypes.c_int32(n_h), _p(a), _p(out))
+    return out
+
+
+def similarity(K) -> np.ndarray:
+    K = _f32(K)
+    S, D = K.shape[-2:]
+    U = K.size // (S * D)
+    out = np.empty(K.shape[:-1], dtype=np.float64)
+    lib().kvmo_similarity(ctypes.c_int64(U), ctypes.c_int32(S), ctypes.c_int32(D), _p(K), _p(out))
+    return out
+
+
+def boundaries(sim: np.ndarray, keep_: np.ndarray, C: int, eps: float, enforce_budget: bool = True):
+    sim = np.ascontiguousarray(sim, dtype=np.float64)
+    keep_ = np.ascontiguousarray(keep_, dtype=np.uint8)
+    S = sim.shape[-1]
+    U = sim.size // S
+    b = np.empty(sim.shape, dtype=np.uint8)
+    fired = np.empty(sim.shape[:-1], dtype=np.int32)
+    lib().kvmo_boundaries(ctypes.c_int64(U), ctypes.c_int32(S), ctypes.c_int32(C), ctypes.c_double(eps),
+                          ctypes.c_int32(1 if enforce_budget else 0), _p(sim), _p(keep_), _p(b), _p(fired))
+    return b, fired
+
+
+def sets(b: np.ndarray, cap: int):
+    b = np.ascontiguousarray(b, dtype=np.uint8)
+    S = b.shape[-1]
+    U = b.size // S
+    lead = b.shape[:-1]
+    set_id = np.empty(b.shape, dtype=np.int32)
+    set_start = np.full(lead + (cap + 1,), -1, dtype=np.int32)
+    out_len = np.empty(lead, dtype=np.int32)
+    lib().kvmo_sets(ctypes.c_int64(U), ctypes.c_int32(S), ctypes.c_int32(cap), _p(b), _p(set_id), _p(set_start),
+                    _p(out_len))
+    return set_id, set_start, out_len
+
+
+def pivots(scores_: np.ndarray, set_start: np.ndarray, out_len: np.ndarray) -> np.ndarray:
+    a = np.ascontiguousarray(scores_, dtype=np.float64)
+    set_start = np.ascontiguousarray(set_start, dtype=np.int32)
+    out_len = np.ascontiguousarray(out_len, dtype=np.int32)
+    S = a.shape[-1]
+    U = a.size // S
+    cap = set_start.shape[-1] - 1
+    pv = np.full(a.shape[:-1] + (cap,), -1, dtype=np.int32)
+    lib().kvmo_pivots(ctypes.c_int64(U), ctypes.c_int32(S), ctypes.c_int32(cap), _p(a), _p(set_start), _p(out_len),
+                      _p(pv))
+    return pv
+
+
+def merge(K, V, set_start, pivot, out_len, sigma: float, scale_v: bool = True, want_weights: bool = False):
+    K, V = _f32(K), _f32(V)
+    set_start = np.ascontiguousarray(set_start, dtype=np.int32)
+    pivot = np.ascontiguousarray(pivot, dtype=np.int32)
+    out_len = np.ascontiguousarray(out_len, dtype=np.int32)
+    S, D = K.shape[-2:]
+    U = K.size // (S * D)
+    cap = set_start.shape[-1] - 1
+    lead = K.shape[:-2]
+    Ko = np.full(lead + (cap, D), np.nan, dtype=np.float64)
+    Vo = np.full(lead + (cap, D), np.nan, dtype=np.float64)
+    w = np.full(lead + (S,), np.nan, dtype=np.float64) if want_weights else None
+    lib().kvmo_merge(ctypes.c_int64(U), ctypes.c_int32(S), ctypes.c_int32(D), ctypes.c_int32(cap),
+                     ctypes.c_double(sigma), ctypes.c_int32(1 if scale_v else 0), _p(K), _p(V), _p(set_start),
+                     _p(pivot), _p(out_len), _p(Ko), _p(Vo), _p(w))
+    return (Ko, Vo, w) if want_weights else (Ko, Vo)
+
+
+@dataclass
+class Compressed:
+    scores: np.ndarray
+    keep: np.ndarray
+    sim: np.ndarray
+    b: np.ndarray
+    set_id: np.ndarray
+    set_start: np.ndarray
+    out_len: np.ndarray
+    pivot: np.ndarray
+    K_out: np.ndarray
+    V_out: np.ndarray
+    cap: int
+    n_r: int
+    n_h: int
+
+
+def compress(Q, K, V, budget: float, recent: float, heavy: float, eps: float = 0.75, sigma: float = 5.0,
+             scale: Optional[float] = None, scale_v: bool = True, enforce_budget: bool = True) -> Compressed:
+    """All steps for one layer through the single C entry point kvmo_compress."""
+    Q, K, V = _f32(Q), _f32(K), _f32(V)
+    B, Hq, S, D = Q.shape
+    Hkv = K.shape[1]
+    if scale is None:
+        scale = 1.0 / math.sqrt(D)
+    C, n_r, n_h = sizes(S, budget, recent, heavy)
+    cap = C if enforce_budget else S
+    lead = (B, Hkv)
+    r = Compressed(
+        scores=np.empty(lead + (S,), np.float64), keep=np.empty(lead + (S,), np.uint8),
+        sim=np.empty(lead + (S,), np.float64), b=np.empty(lead + (S,), np.uint8),
+        set_id=np.empty(lead + (S,), np.int32), set_start=np.full(lead + (cap + 1,), -1, np.int32),
+        out_len=np.empty(lead, np.int32), pivot=np.full(lead + (cap,), -1, np.int32),
+        K_out=np.full(lead + (cap, D), np.nan, np.float64), V_out=np.full(lead + (cap, D), np.nan, np.float64),
+        cap=cap, n_r=n_r, n_h=n_h)
+    lib().kvmo_compress(ctypes.c_int32(B), ctypes.c_int32(Hq), ctypes.c_int32(Hkv), ctypes.c_int32(S),
+                        ctypes.c_int32(D), ctypes.c_double(scale), ctypes.c_int32(cap), ctypes.c_int32(n_r),
+                        ctypes.c_int32(n_h), ctypes.c_double(eps), ctypes.c_double(sigma),
+                        ctypes.c_int32(1 if scale_v else 0), ctypes.c_int32(1 if enforce_budget else 0),
+                        _p(Q), _p(K), _p(V), _p(r.scores), _p(r.keep), _p(r.sim), _p(r.b), _p(r.set_id),
+                        _p(r.set_start), _p(r.out_len), _p(r.pivot), _p(r.K_out), _p(r.V_out))
+    return r
