@@ -1,0 +1,174 @@
+/*
+ * kvm -- prefill-time KV-cache compression by adaptive merging (KVMerger,
+ * arXiv 2407.08454) for NVIDIA B200 (sm_100a).  C ABI.
+ *
+ * Per attention layer and per (batch entry, KV head) "unit" the library
+ *   1. sums the causal attention map softmax(Q K^T * scale) over queries, giving
+ *      one aggregated score per key (Eq. 1; Algorithm 2; Eq. 6; for grouped-query
+ *      attention the maps of a KV head's query heads are averaged, Section 5.2);
+ *   2. measures the cosine similarity of neighbouring keys (Eq. 2) and cuts the
+ *      sequence into merging sets of consecutive tokens (Algorithm 1,
+ *      Definition 4.1); the most recent tokens and the keys with the largest
+ *      scores are conserved, i.e. never merged (Sections 4.1, 4.2, 5.1);
+ *   3. picks each set's pivot, the key with the largest score (Eq. 6);
+ *   4. merges each set's keys and values into one state with Gaussian-kernel
+ *      weights around the pivot (Eq. 4, Eq. 5, Definition 4.2) and writes the
+ *      states densely, in token order.
+ *
+ * Conventions for every entry point
+ *   - Unless a parameter says "host", tensor pointers are DEVICE pointers owned by
+ *     the caller, contiguous row-major in the stated shape and 16-byte aligned.
+ *     Inputs are never written.
+ *   - The library allocates no memory and keeps no state between calls.  Scratch
+ *     space is the caller's `ws` buffer of at least kvm_workspace_bytes() bytes;
+ *     its contents are undefined afterwards.  Calls that share a workspace must
+ *     be ordered on one stream.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL is
+ *     the legacy default stream) and the call returns without synchronising.
+ *   - Return value: KVM_OK, or a negative kvm_status found on the host before
+ *     anything was enqueued (KVM_E_CUDA: a launch or copy was refused by the
+ *     runtime).  Conditions found on the device are reported through kvm_stats.
+ *   - U = batch * n_kv_heads units; G = n_q_heads / n_kv_heads; S = seq;
+ *     D = head_dim; cap = output capacity in rows per unit =
+ *     floor(budget * S) when enforce_budget, else S.
+ */
+#ifndef KVM_H_
+#define KVM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define KVM_VERSION 100
+
+enum kvm_dtype { KVM_BF16 = 0, KVM_F32 = 1 };
+
+enum kvm_status {
+    KVM_OK = 0,
+    KVM_E_NULL = -1,        /* a required pointer is NULL */
+    KVM_E_SHAPE = -2,       /* sizes not positive, heads not divisible, head_dim not 64/128, seq too long */
+    KVM_E_DTYPE = -3,       /* dtype is not a kvm_dtype */
+    KVM_E_PARAM = -4,       /* ratio/threshold/bandwidth out of range, or capacity too small for the conserved set */
+    KVM_E_ALIGN = -5,       /* a tensor pointer is not 16-byte aligned */
+    KVM_E_WORKSPACE = -6,   /* ws is NULL or smaller than kvm_workspace_bytes() */
+    KVM_E_UNSUPPORTED = -7, /* valid request this build cannot run (e.g. non-causal) */
+    KVM_E_CUDA = -8,        /* the CUDA runtime refused a launch, a copy or a driver lookup */
+    KVM_E_DEVICE_TIMEOUT = -9 /* only ever appears in kvm_stats.status: a bounded device wait gave up */
+};
+
+/* The paper's problem statement as a plain struct (Section 2.4; hyper-parameters of Section 5.1). */
+typedef struct kvm_params {
+    int32_t batch, n_q_heads, n_kv_heads, seq, head_dim; /* head_dim 64 or 128; seq <= KVM_MAX_SEQ */
+    int32_t dtype;               /* kvm_dtype of Q, K, V and of K_out, V_out */
+    float budget;                /* (0,1]: cache budget, 0.50 or 0.35 in the paper */
+    float recent_ratio;          /* share of S conserved as most recent tokens; < 0: preset 0.17 (budget >= 0.425) else 0.08 */
+    float heavy_ratio;           /* share of S conserved for largest scores;    < 0: preset 0.12 (budget >= 0.425) else 0.02 */
+    float sim_threshold;         /* epsilon of Algorithm 1; neighbours group when similarity > epsilon (strict); paper: 0.75 */
+    float sigma;                 /* Gaussian bandwidth of Eq. 4, > 0; the paper's best fixed value is 5 */
+    float softmax_scale;         /* <= 0: 1/sqrt(head_dim) as in Eq. 1 */
+    int32_t causal;              /* must be 1 */
+    int32_t scale_v_by_set_size; /* 1: value weights are multiplied by the set size (text after Eq. 5); 0: plain weighted mean */
+    int32_t enforce_budget;      /* 1: at most floor(budget*S) sets per unit (see kvm_segment); 0: capacity is S */
+} kvm_params;
+
+#define KVM_MAX_SEQ 65536
+
+/* Device-side report, filled by kvm_segment / kvm_compress when given.  Zero it before the call. */
+typedef struct kvm_stats {
+    int32_t status;            /* KVM_OK or KVM_E_DEVICE_TIMEOUT */
+    int32_t units_budget_rule; /* units in which the budget rule removed boundaries */
+    int32_t near_threshold;    /* neighbour pairs with |similarity - epsilon| < 1e-3 */
+    int32_t min_out_len, max_out_len; /* over units (min starts at 0 meaning "unset") */
+    int64_t sum_out_len;
+} kvm_stats;
+
+/* Derived sizes for a parameter set: capacity rows per unit, recent count, heavy-hitter count. Host only. */
+int kvm_sizes(const kvm_params* p, int32_t* cap, int32_t* n_recent, int32_t* n_heavy);
+
+/* Bytes of scratch every entry point below accepts for these parameters. Host only. */
+int kvm_workspace_bytes(const kvm_params* p, size_t* bytes);
+
+/*
+ * Aggregated attention scores (Eq. 1 restricted to the causal part; column sums
+ * as in Algorithm 2 / Eq. 6; mean over the G query heads of a KV head, Section 5.2).
+ *   Q [batch, n_q_heads, S, D], K [batch, n_kv_heads, S, D] in p->dtype.
+ *   lse_in: NULL, or [batch, n_q_heads, S] fp32 natural-log row log-sum-exp of
+ *           the scaled causal logits (e.g. from the prefill attention kernel);
+ *           when given, the row pass is skipped.
+ *   scores: [batch, n_kv_heads, S] fp32, written.
+ * bf16 runs on tensor cores with fp32 accumulation and fp32 softmax; fp32 runs in fp32 FMA.
+ */
+int kvm_score(const kvm_params* p, const void* Q, const void* K, const float* lse_in,
+              float* scores, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Merging-set identification and pivots (Eq. 2, Algorithm 1, Definition 4.1, Eq. 6).
+ *   K [batch, n_kv_heads, S, D]; scores [batch, n_kv_heads, S] fp32.
+ *   Conserved tokens: the last n_recent positions and, among the others, the
+ *   n_heavy largest scores (ties: lower index).  Token j starts a set when j = 0,
+ *   when j or j-1 is conserved, or when cos(k_{j-1}, k_j) > epsilon is false.
+ *   Budget rule (enforce_budget): if that gives more than cap sets, only the
+ *   cap - (forced cuts) similarity cuts with the smallest similarity are kept
+ *   (ties: lower index), which equals lowering epsilon for that unit.
+ *   Outputs (all written for rows < out_len only):
+ *     set_id    NULL or [U, S] i32     set index of each token
+ *     set_start [U, cap+1] i32         first token of each set; set_start[out_len] = S
+ *     pivot     [U, cap] i32           token with the largest score in the set (ties: lowest index)
+ *     out_len   [U] i32                number of sets
+ *     sim_out   NULL or [U, S] fp32    cos(k_{j-1}, k_j), entry 0 is 0
+ *     stats     NULL or device kvm_stats
+ */
+int kvm_segment(const kvm_params* p, const void* K, const float* scores,
+                int32_t* set_id, int32_t* set_start, int32_t* pivot, int32_t* out_len,
+                float* sim_out, kvm_stats* stats, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Gaussian-kernel weighted merge and compaction (Eq. 4 with fixed sigma, Eq. 5,
+ * Definition 4.2, Algorithm 2).  For set s with tokens [set_start[s], set_start[s+1])
+ * and pivot p:  g_j = exp(-|k_p - k_j|^2 / (2 sigma^2)),  K_out[s] = sum g_j k_j / sum g_j,
+ * V_out[s] = n_s * sum g_j v_j / sum g_j (n_s omitted when !scale_v_by_set_size).
+ * fp32 accumulation, one round-to-nearest-even conversion at the store; a set of
+ * one token is copied bit for bit.
+ *   K, V [U, S, D]; set_start [U, cap+1]; pivot [U, cap]; out_len [U] (device).
+ *   K_out, V_out [U, cap, D] in p->dtype; rows >= out_len are left untouched.
+ *   out_size: NULL or [U, cap] i32, the size of each set.
+ */
+int kvm_merge_compact(const kvm_params* p, const void* K, const void* V,
+                      const int32_t* set_start, const int32_t* pivot, const int32_t* out_len,
+                      void* K_out, void* V_out, int32_t* out_size,
+                      void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * The whole path for one layer: kvm_score, kvm_segment, kvm_merge_compact chained
+ * on the stream with intermediates in the workspace.
+ *   out_pos    [U, cap] i32   pivot token index of each output row (ascending)
+ *   scores_out NULL or [U, S] fp32
+ *   stats      NULL or device kvm_stats
+ */
+int kvm_compress(const kvm_params* p, const void* Q, const void* K, const void* V,
+                 void* K_out, void* V_out, int32_t* out_len, int32_t* out_pos,
+                 float* scores_out, kvm_stats* stats, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * kvm_compress for callers whose tensors live in HOST memory (pinned memory
+ * makes the copies asynchronous).  Q, K, V, K_out, V_out, out_len, out_pos are
+ * host pointers with the shapes of kvm_compress; `dev` is a caller-owned device
+ * buffer of at least kvm_host_staging_bytes() bytes that holds the staged tensors
+ * and the workspace.  Copies in, compresses, copies all cap rows out; everything
+ * is enqueued on the stream and the caller synchronises before reading.
+ */
+int kvm_host_staging_bytes(const kvm_params* p, size_t* bytes);
+int kvm_compress_host(const kvm_params* p, const void* Q, const void* K, const void* V,
+                      void* K_out, void* V_out, int32_t* out_len, int32_t* out_pos,
+                      void* dev, size_t dev_bytes, void* cuda_stream);
+
+const char* kvm_status_string(int status);
+int kvm_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KVM_H_ */

@@ -1,0 +1,250 @@
+// C ABI of the kvm library: host-side validation, workspace carving, dispatch.
+// All checks run before anything is enqueued; nothing here allocates or synchronises.
+#include <math.h>
+#include <string.h>
+
+#include "common.cuh"
+
+namespace kvm {
+namespace {
+
+inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+
+int derive(const kvm_params* p, Dims& d) {
+    if (!p) return KVM_E_NULL;
+    if (p->dtype != KVM_BF16 && p->dtype != KVM_F32) return KVM_E_DTYPE;
+    if (p->batch < 1 || p->n_q_heads < 1 || p->n_kv_heads < 1 || p->seq < 1) return KVM_E_SHAPE;
+    if (p->n_q_heads % p->n_kv_heads != 0) return KVM_E_SHAPE;
+    if (p->head_dim != 64 && p->head_dim != 128) return KVM_E_SHAPE;
+    if (p->seq > KVM_MAX_SEQ) return KVM_E_SHAPE;
+    if ((long long)p->batch * p->n_q_heads > 65535) return KVM_E_SHAPE;
+    if (!(p->budget > 0.f && p->budget <= 1.f)) return KVM_E_PARAM;
+    if (!(p->sigma > 0.f) || !isfinite(p->sigma)) return KVM_E_PARAM;
+    if (!isfinite(p->sim_threshold)) return KVM_E_PARAM;
+    if (!isfinite(p->softmax_scale)) return KVM_E_PARAM;
+    if (p->causal != 1) return KVM_E_UNSUPPORTED;
+    const bool half_budget = p->budget >= 0.425f;
+    const float recent = p->recent_ratio < 0.f ? (half_budget ? 0.17f : 0.08f) : p->recent_ratio;
+    const float heavy = p->heavy_ratio < 0.f ? (half_budget ? 0.12f : 0.02f) : p->heavy_ratio;
+    if (!(recent >= 0.f && recent <= 1.f) || !(heavy >= 0.f && heavy <= 1.f)) return KVM_E_PARAM;
+    d.B = p->batch; d.Hq = p->n_q_heads; d.Hkv = p->n_kv_heads; d.G = d.Hq / d.Hkv;
+    d.S = p->seq; d.D = p->head_dim; d.U = d.B * d.Hkv; d.dtype = p->dtype;
+    const int C = (int)floor((double)p->budget * (double)d.S);
+    d.n_r = (int)floor((double)recent * (double)d.S);
+    d.n_h = (int)floor((double)heavy * (double)d.S);
+    d.enforce = p->enforce_budget ? 1 : 0;
+    d.cap = d.enforce ? C : d.S;
+    // the forced cuts alone (first token, recent window, each heavy hitter and its right neighbour) must fit
+    if (d.enforce && (long long)d.cap < 1LL + d.n_r + 2LL * d.n_h) return KVM_E_PARAM;
+    if (d.cap < 1) return KVM_E_PARAM;
+    d.scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)d.D);
+    d.eps = p->sim_threshold;
+    d.sigma = p->sigma;
+    d.scale_v = p->scale_v_by_set_size ? 1 : 0;
+    return KVM_OK;
+}
+
+struct Workspace {
+    int* counters;      // 64 ints
+    float* lse;         // [B,Hq,S]
+    float* scores;      // [U,S]
+    float* sim;         // [U,S]
+    int32_t* set_start; // [U,cap+1]
+    size_t bytes;
+};
+
+Workspace carve(const Dims& d, void* base) {
+    Workspace w;
+    size_t off = 0;
+    auto take = [&](size_t n) { size_t o = off; off += align_up(n); return (char*)base + o; };
+    w.counters = (int*)take(64 * sizeof(int));
+    w.lse = (float*)take((size_t)d.B * d.Hq * d.S * sizeof(float));
+    w.scores = (float*)take((size_t)d.U * d.S * sizeof(float));
+    w.sim = (float*)take((size_t)d.U * d.S * sizeof(float));
+    w.set_start = (int32_t*)take((size_t)d.U * (d.cap + 1) * sizeof(int32_t));
+    w.bytes = off;
+    return w;
+}
+
+inline bool misaligned(const void* p) { return ((uintptr_t)p & 15u) != 0; }
+
+int check_ws(const Dims& d, void* ws, size_t ws_bytes, Workspace& w) {
+    if (!ws) return KVM_E_WORKSPACE;
+    if (misaligned(ws)) return KVM_E_ALIGN;
+    w = carve(d, ws);
+    if (ws_bytes < w.bytes) return KVM_E_WORKSPACE;
+    return KVM_OK;
+}
+
+cudaError_t run_score(const Dims& d, const void* Q, const void* K, const float* lse_in, float* scores,
+                      const Workspace& w, kvm_stats* stats, cudaStream_t st) {
+    (void)stats;
+    return launch_score_simt(d, Q, K, lse_in, w.lse, scores, st);
+}
+
+}  // namespace
+}  // namespace kvm
+
+using namespace kvm;
+
+extern "C" {
+
+int kvm_version(void) { return KVM_VERSION; }
+
+const char* kvm_status_string(int s) {
+    switch (s) {
+        case KVM_OK: return "ok";
+        case KVM_E_NULL: return "a required pointer is NULL";
+        case KVM_E_SHAPE: return "unsupported shape";
+        case KVM_E_DTYPE: return "unknown dtype";
+        case KVM_E_PARAM: return "parameter out of range or capacity too small for the conserved tokens";
+        case KVM_E_ALIGN: return "pointer not 16-byte aligned";
+        case KVM_E_WORKSPACE: return "workspace missing or too small";
+        case KVM_E_UNSUPPORTED: return "unsupported request";
+        case KVM_E_CUDA: return "CUDA runtime error";
+        case KVM_E_DEVICE_TIMEOUT: return "a bounded device-side wait gave up";
+        default: return "unknown status";
+    }
+}
+
+int kvm_sizes(const kvm_params* p, int32_t* cap, int32_t* n_recent, int32_t* n_heavy) {
+    Dims d;
+    const int rc = derive(p, d);
+    if (rc != KVM_OK) return rc;
+    if (cap) *cap = d.cap;
+    if (n_recent) *n_recent = d.n_r;
+    if (n_heavy) *n_heavy = d.n_h;
+    return KVM_OK;
+}
+
+int kvm_workspace_bytes(const kvm_params* p, size_t* bytes) {
+    Dims d;
+    const int rc = derive(p, d);
+    if (rc != KVM_OK) return rc;
+    if (!bytes) return KVM_E_NULL;
+    *bytes = carve(d, nullptr).bytes;
+    return KVM_OK;
+}
+
+int kvm_score(const kvm_params* p, const void* Q, const void* K, const float* lse_in, float* scores, void* ws,
+              size_t ws_bytes, void* cuda_stream) {
+    Dims d;
+    int rc = derive(p, d);
+    if (rc != KVM_OK) return rc;
+    if (!Q || !K || !scores) return KVM_E_NULL;
+    if (misaligned(Q) || misaligned(K) || misaligned(scores) || (lse_in && misaligned(lse_in))) return KVM_E_ALIGN;
+    Workspace w;
+    if ((rc = check_ws(d, ws, ws_bytes, w)) != KVM_OK) return rc;
+    return run_score(d, Q, K, lse_in, scores, w, nullptr, (cudaStream_t)cuda_stream) == cudaSuccess ? KVM_OK
+                                                                                                    : KVM_E_CUDA;
+}
+
+int kvm_segment(const kvm_params* p, const void* K, const float* scores, int32_t* set_id, int32_t* set_start,
+                int32_t* pivot, int32_t* out_len, float* sim_out, kvm_stats* stats, void* ws, size_t ws_bytes,
+                void* cuda_stream) {
+    Dims d;
+    int rc = derive(p, d);
+    if (rc != KVM_OK) return rc;
+    if (!K || !scores || !set_start || !pivot || !out_len) return KVM_E_NULL;
+    if (misaligned(K) || misaligned(scores)) return KVM_E_ALIGN;
+    Workspace w;
+    if ((rc = check_ws(d, ws, ws_bytes, w)) != KVM_OK) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    float* sim = sim_out ? sim_out : w.sim;
+    if (launch_similarity(d, K, sim, st) != cudaSuccess) return KVM_E_CUDA;
+    if (launch_segment(d, scores, sim, set_id, set_start, pivot, out_len, stats, st) != cudaSuccess)
+        return KVM_E_CUDA;
+    return KVM_OK;
+}
+
+int kvm_merge_compact(const kvm_params* p, const void* K, const void* V, const int32_t* set_start,
+                      const int32_t* pivot, const int32_t* out_len, void* K_out, void* V_out, int32_t* out_size,
+                      void* ws, size_t ws_bytes, void* cuda_stream) {
+    Dims d;
+    int rc = derive(p, d);
+    if (rc != KVM_OK) return rc;
+    if (!K || !V || !set_start || !pivot || !out_len || !K_out || !V_out) return KVM_E_NULL;
+    if (misaligned(K) || misaligned(V) || misaligned(K_out) || misaligned(V_out)) return KVM_E_ALIGN;
+    Workspace w;
+    if ((rc = check_ws(d, ws, ws_bytes, w)) != KVM_OK) return rc;
+    return launch_merge(d, K, V, set_start, pivot, out_len, K_out, V_out, out_size, (cudaStream_t)cuda_stream) ==
+                   cudaSuccess
+               ? KVM_OK
+               : KVM_E_CUDA;
+}
+
+int kvm_compress(const kvm_params* p, const void* Q, const void* K, const void* V, void* K_out, void* V_out,
+                 int32_t* out_len, int32_t* out_pos, float* scores_out, kvm_stats* stats, void* ws,
+                 size_t ws_bytes, void* cuda_stream) {
+    Dims d;
+    int rc = derive(p, d);
+    if (rc != KVM_OK) return rc;
+    if (!Q || !K || !V || !K_out || !V_out || !out_len || !out_pos) return KVM_E_NULL;
+    if (misaligned(Q) || misaligned(K) || misaligned(V) || misaligned(K_out) || misaligned(V_out) ||
+        (scores_out && misaligned(scores_out)))
+        return KVM_E_ALIGN;
+    Workspace w;
+    if ((rc = check_ws(d, ws, ws_bytes, w)) != KVM_OK) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    float* scores = scores_out ? scores_out : w.scores;
+    if (run_score(d, Q, K, nullptr, scores, w, stats, st) != cudaSuccess) return KVM_E_CUDA;
+    if (launch_similarity(d, K, w.sim, st) != cudaSuccess) return KVM_E_CUDA;
+    if (launch_segment(d, scores, w.sim, nullptr, w.set_start, out_pos, out_len, stats, st) != cudaSuccess)
+        return KVM_E_CUDA;
+    if (launch_merge(d, K, V, w.set_start, out_pos, out_len, K_out, V_out, nullptr, st) != cudaSuccess)
+        return KVM_E_CUDA;
+    return KVM_OK;
+}
+
+int kvm_host_staging_bytes(const kvm_params* p, size_t* bytes) {
+    Dims d;
+    const int rc = derive(p, d);
+    if (rc != KVM_OK) return rc;
+    if (!bytes) return KVM_E_NULL;
+    const size_t e = d.dtype == KVM_BF16 ? 2 : 4;
+    size_t off = 0;
+    off += align_up((size_t)d.B * d.Hq * d.S * d.D * e);        // Q
+    off += 2 * align_up((size_t)d.U * d.S * d.D * e);           // K, V
+    off += 2 * align_up((size_t)d.U * d.cap * d.D * e);         // K_out, V_out
+    off += align_up((size_t)d.U * sizeof(int32_t));             // out_len
+    off += align_up((size_t)d.U * d.cap * sizeof(int32_t));     // out_pos
+    off += carve(d, nullptr).bytes;
+    *bytes = off;
+    return KVM_OK;
+}
+
+int kvm_compress_host(const kvm_params* p, const void* Q, const void* K, const void* V, void* K_out, void* V_out,
+                      int32_t* out_len, int32_t* out_pos, void* dev, size_t dev_bytes, void* cuda_stream) {
+    Dims d;
+    int rc = derive(p, d);
+    if (rc != KVM_OK) return rc;
+    if (!Q || !K || !V || !K_out || !V_out || !out_len || !out_pos) return KVM_E_NULL;
+    size_t need = 0;
+    kvm_host_staging_bytes(p, &need);
+    if (!dev || dev_bytes < need) return KVM_E_WORKSPACE;
+    if (misaligned(dev)) return KVM_E_ALIGN;
+    const size_t e = d.dtype == KVM_BF16 ? 2 : 4;
+    const size_t nQ = (size_t)d.B * d.Hq * d.S * d.D * e, nK = (size_t)d.U * d.S * d.D * e;
+    const size_t nO = (size_t)d.U * d.cap * d.D * e, nL = (size_t)d.U * sizeof(int32_t);
+    const size_t nP = (size_t)d.U * d.cap * sizeof(int32_t);
+    char* b = (char*)dev;
+    size_t off = 0;
+    auto take = [&](size_t n) { char* q = b + off; off += align_up(n); return q; };
+    char* dQ = take(nQ); char* dK = take(nK); char* dV = take(nK);
+    char* dKo = take(nO); char* dVo = take(nO); char* dL = take(nL); char* dP = take(nP);
+    char* ws = b + off;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (cudaMemcpyAsync(dQ, Q, nQ, cudaMemcpyHostToDevice, st) != cudaSuccess) return KVM_E_CUDA;
+    if (cudaMemcpyAsync(dK, K, nK, cudaMemcpyHostToDevice, st) != cudaSuccess) return KVM_E_CUDA;
+    if (cudaMemcpyAsync(dV, V, nK, cudaMemcpyHostToDevice, st) != cudaSuccess) return KVM_E_CUDA;
+    rc = kvm_compress(p, dQ, dK, dV, dKo, dVo, (int32_t*)dL, (int32_t*)dP, nullptr, nullptr, ws, dev_bytes - off,
+                      cuda_stream);
+    if (rc != KVM_OK) return rc;
+    if (cudaMemcpyAsync(K_out, dKo, nO, cudaMemcpyDeviceToHost, st) != cudaSuccess) return KVM_E_CUDA;
+    if (cudaMemcpyAsync(V_out, dVo, nO, cudaMemcpyDeviceToHost, st) != cudaSuccess) return KVM_E_CUDA;
+    if (cudaMemcpyAsync(out_len, dL, nL, cudaMemcpyDeviceToHost, st) != cudaSuccess) return KVM_E_CUDA;
+    if (cudaMemcpyAsync(out_pos, dP, nP, cudaMemcpyDeviceToHost, st) != cudaSuccess) return KVM_E_CUDA;
+    return KVM_OK;
+}
+
+}  // extern "C"

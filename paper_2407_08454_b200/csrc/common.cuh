@@ -1,0 +1,62 @@
+// Shared declarations of the kvm CUDA library (internal; the public ABI is include/kvm.h).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "kvm.h"
+
+namespace kvm {
+
+// Validated, derived problem sizes handed to every launcher.
+struct Dims {
+    int B, Hq, Hkv, G, S, D, U;
+    int cap, n_r, n_h;
+    int dtype;  // kvm_dtype
+    float scale, eps, sigma;
+    int scale_v, enforce;
+};
+
+// 16-byte vector <-> fp32 lanes.  Vec<T>::N elements of T per 16 bytes.
+template <typename T> struct Vec;
+template <> struct Vec<float> {
+    static constexpr int N = 4;
+    static __device__ __forceinline__ void unpack(const uint4& r, float* f) {
+        f[0] = __uint_as_float(r.x); f[1] = __uint_as_float(r.y);
+        f[2] = __uint_as_float(r.z); f[3] = __uint_as_float(r.w);
+    }
+    static __device__ __forceinline__ uint4 pack(const float* f) {
+        return make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]), __float_as_uint(f[3]));
+    }
+};
+template <> struct Vec<__nv_bfloat16> {
+    static constexpr int N = 8;
+    static __device__ __forceinline__ void unpack(const uint4& r, float* f) {
+        // bf16 -> fp32 is a 16-bit left shift
+        f[0] = __uint_as_float(r.x << 16); f[1] = __uint_as_float(r.x & 0xffff0000u);
+        f[2] = __uint_as_float(r.y << 16); f[3] = __uint_as_float(r.y & 0xffff0000u);
+        f[4] = __uint_as_float(r.z << 16); f[5] = __uint_as_float(r.z & 0xffff0000u);
+        f[6] = __uint_as_float(r.w << 16); f[7] = __uint_as_float(r.w & 0xffff0000u);
+    }
+    static __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+        __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);  // round to nearest even
+        return *reinterpret_cast<uint32_t*>(&v);
+    }
+    static __device__ __forceinline__ uint4 pack(const float* f) {
+        return make_uint4(pack2(f[0], f[1]), pack2(f[2], f[3]), pack2(f[4], f[5]), pack2(f[6], f[7]));
+    }
+};
+
+__device__ __forceinline__ uint4 ldg16(const void* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
+
+// Launchers (each enqueues on the stream and returns the launch status).
+cudaError_t launch_score_simt(const Dims& d, const void* Q, const void* K, const float* lse_in, float* lse_ws,
+                              float* scores, cudaStream_t st);
+cudaError_t launch_similarity(const Dims& d, const void* K, float* sim, cudaStream_t st);
+cudaError_t launch_segment(const Dims& d, const float* scores, const float* sim, int32_t* set_id,
+                           int32_t* set_start, int32_t* pivot, int32_t* out_len, kvm_stats* stats, cudaStream_t st);
+cudaError_t launch_merge(const Dims& d, const void* K, const void* V, const int32_t* set_start,
+                         const int32_t* pivot, const int32_t* out_len, void* K_out, void* V_out,
+                         int32_t* out_size, cudaStream_t st);
+
+}  // namespace kvm
