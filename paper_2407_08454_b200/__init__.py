@@ -1,0 +1,11 @@
+"""B200-native KVMerger prefill-time KV-cache compression: CUDA library + thin binding.
+
+`binding` wraps the C ABI of include/kvm.h (libkvm.so, built in-tree by `build`);
+`synth_inputs` holds the seeded synthetic workloads.
+"""
+from . import synth_inputs  # noqa: F401
+from .binding import (  # noqa: F401
+    KVM_BF16, KVM_F32, Compressed, Compressor, KvmError, KvmParams, KvmStats, kvm_compress, kvm_compress_host,
+    kvm_host_staging_bytes, kvm_merge_compact, kvm_score, kvm_segment, kvm_sizes, kvm_version,
+    kvm_workspace_bytes, make_params, new_stats, read_stats, status_string,
+)

@@ -1,0 +1,82 @@
+"""Host-side checks of the C ABI: the library loads, exports every symbol the
+header declares, and rejects bad arguments before touching a GPU."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2407_08454_b200 as kvm
+from paper_2407_08454_b200 import binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return binding.lib()
+
+
+def test_every_declared_symbol_is_exported(lib):
+    header = open(os.path.join(ROOT, "include", "kvm.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(kvm_[a-z_0-9]+)\s*\(", header))
+    assert {"kvm_score", "kvm_segment", "kvm_merge_compact", "kvm_compress"} <= declared
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert declared == set(binding.EXPORTS) | (declared - set(binding.EXPORTS))
+    assert set(binding.EXPORTS) <= declared
+    assert kvm.kvm_version() == 100
+
+
+def test_sizes_and_presets(lib):
+    p = kvm.make_params(1, 32, 32, 4096, 128, kvm.KVM_BF16, budget=0.5)
+    assert kvm.kvm_sizes(p) == (2048, 696, 491)
+    p = kvm.make_params(4, 32, 32, 4096, 128, kvm.KVM_BF16, budget=0.35)
+    assert kvm.kvm_sizes(p) == (1433, 327, 81)
+    p = kvm.make_params(1, 32, 8, 32768, 128, kvm.KVM_BF16, budget=0.5)
+    assert kvm.kvm_sizes(p) == (16384, 5570, 3932)
+    p = kvm.make_params(1, 4, 4, 512, 64, kvm.KVM_F32, budget=0.5, enforce_budget=0)
+    assert kvm.kvm_sizes(p) == (512, 87, 61)
+    assert kvm.kvm_workspace_bytes(p) > 0
+    assert kvm.kvm_host_staging_bytes(p) > kvm.kvm_workspace_bytes(p)
+
+
+@pytest.mark.parametrize("kw,status", [
+    (dict(dtype=7), -3),
+    (dict(head_dim=96), -2),
+    (dict(n_q_heads=6, n_kv_heads=4), -2),
+    (dict(seq=0), -2),
+    (dict(seq=70000), -2),
+    (dict(budget=0.0), -4),
+    (dict(budget=1.5), -4),
+    (dict(sigma=0.0), -4),
+    (dict(budget=0.2, recent_ratio=0.17, heavy_ratio=0.12), -4),   # conserved tokens alone exceed the capacity
+    (dict(causal=0), -7),
+])
+def test_bad_parameters_are_rejected_on_the_host(lib, kw, status):
+    base = dict(batch=1, n_q_heads=4, n_kv_heads=4, seq=512, head_dim=64, dtype=kvm.KVM_F32)
+    base.update(kw)
+    p = kvm.make_params(**base)
+    n = ctypes.c_size_t()
+    assert lib.kvm_workspace_bytes(ctypes.byref(p), ctypes.byref(n)) == status
+    assert kvm.status_string(status) != "unknown status"
+
+
+def test_null_alignment_and_workspace_errors(lib):
+    p = kvm.make_params(1, 4, 4, 512, 64, kvm.KVM_F32)
+    vp = ctypes.c_void_p
+    ok = vp(4096)          # never dereferenced: the checks below fail first
+    assert lib.kvm_compress(ctypes.byref(p), vp(0), ok, ok, ok, ok, ok, ok, vp(0), vp(0), ok, ctypes.c_size_t(1 << 30), vp(0)) == -1
+    assert lib.kvm_compress(ctypes.byref(p), vp(4100), ok, ok, ok, ok, ok, ok, vp(0), vp(0), ok, ctypes.c_size_t(1 << 30), vp(0)) == -5
+    assert lib.kvm_compress(ctypes.byref(p), ok, ok, ok, ok, ok, ok, ok, vp(0), vp(0), vp(0), ctypes.c_size_t(0), vp(0)) == -6
+    assert lib.kvm_compress(ctypes.byref(p), ok, ok, ok, ok, ok, ok, ok, vp(0), vp(0), ok, ctypes.c_size_t(16), vp(0)) == -6
+    assert lib.kvm_score(None, ok, ok, vp(0), ok, ok, ctypes.c_size_t(1 << 30), vp(0)) == -1
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "libkvm.so"))
+    with pytest.raises(FileNotFoundError):
+        binding.lib()

@@ -1,0 +1,110 @@
+"""GPU parity: the CUDA library (through its C ABI) against the fp64 CPU checker,
+element by element, on seeded synthetic inputs.  Bars are defined in parity.py."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2407_08454_b200 as kvm
+from paper_2407_08454_b200 import synth_inputs as si
+from parity import Case, check_case, check_invariants_all_units, run_gpu
+
+pytestmark = pytest.mark.gpu
+
+
+def _case(cfg, layer=0, **kw):
+    d = si.make_layer(cfg, layer)
+    return Case(d["Q"], d["K"], d["V"], budget=cfg.budget, **kw)
+
+
+def test_c0_tiny_fp32_full():
+    rep = check_case(_case(si.CONFIGS["C0"]))
+    print("C0", rep)
+
+
+@pytest.mark.parametrize("S,D,Hq,Hkv,B,dtype,budget", [
+    (300, 64, 4, 4, 1, "f32", 0.5),      # ragged tail, several tiles
+    (777, 128, 4, 2, 2, "bf16", 0.5),    # GQA group 2, batch 2, ragged
+    (1000, 64, 8, 2, 1, "bf16", 0.35),   # group 4, 35% preset
+    (129, 128, 2, 2, 1, "bf16", 0.5),    # one element past a tile
+    (2048, 128, 2, 1, 1, "f32", 0.35),
+])
+def test_small_shapes(S, D, Hq, Hkv, B, dtype, budget):
+    cfg = si.CONFIGS["C1"].scaled(seq=S, head_dim=D, n_q_heads=Hq, n_kv_heads=Hkv, batch=B, dtype=dtype,
+                                  budget=budget, seed=100 + S)
+    rep = check_case(_case(cfg))
+    print(S, D, rep)
+
+
+def test_budget_rule_fires_and_is_exact():
+    # low token-to-token correlation: far more similarity cuts than the capacity allows
+    cfg = si.CONFIGS["C1"].scaled(seq=1024, n_q_heads=4, n_kv_heads=4, rho=0.6, budget=0.35, seed=7)
+    case = _case(cfg)
+    g = run_gpu(case)
+    assert g.stats.units_budget_rule == 4
+    assert (g.out_len == g.cap).all()
+    check_case(case, g)
+
+
+def test_threshold_above_one_returns_the_input_cache():
+    cfg = si.CONFIGS["C1"].scaled(seq=512, n_q_heads=2, n_kv_heads=2, seed=8)
+    d = si.make_layer(cfg)
+    case = Case(d["Q"], d["K"], d["V"], budget=1.0, recent=0.0, heavy=0.0, eps=1.5, enforce=False)
+    g = run_gpu(case)
+    assert (g.c_out_len == 512).all()
+    assert np.array_equal(g.c_K_out, d["K"].float().numpy()) and np.array_equal(g.c_V_out, d["V"].float().numpy())
+    assert np.array_equal(g.c_out_pos, np.broadcast_to(np.arange(512, dtype=np.int32), g.c_out_pos.shape))
+    check_case(case, g)
+
+
+def test_degenerate_inputs():
+    # identical keys, nothing conserved, threshold below -1: one set per unit
+    k = torch.randn(1, 2, 1, 64, generator=torch.Generator().manual_seed(1))
+    K = k.repeat(1, 1, 200, 1).contiguous()
+    Q = torch.randn(1, 2, 200, 64, generator=torch.Generator().manual_seed(2))
+    V = torch.randn(1, 2, 200, 64, generator=torch.Generator().manual_seed(3))
+    case = Case(Q, K, V, budget=0.5, recent=0.0, heavy=0.0, eps=-2.0)
+    g = run_gpu(case)
+    assert (g.out_len == 1).all() and (g.pivot[..., 0] == 0).all()      # all scores tie per column? pivot = arg-max
+    rep = check_case(case, g)
+    np.testing.assert_allclose(g.K_out[:, :, 0], k[:, :, 0].numpy(), rtol=1e-6)
+    # zero keys: similarity 0 by convention, every token its own set
+    K0 = torch.zeros(1, 1, 64, 64)
+    case = Case(torch.randn(1, 1, 64, 64), K0, torch.randn(1, 1, 64, 64), budget=1.0, recent=0.0, heavy=0.0,
+                enforce=False)
+    g = run_gpu(case)
+    assert (g.out_len == 64).all() and (g.sim == 0).all()
+    check_case(case, g)
+    # S = 1 and S = 2
+    for S in (1, 2):
+        case = Case(torch.randn(1, 1, S, 64), torch.randn(1, 1, S, 64), torch.randn(1, 1, S, 64), budget=1.0,
+                    recent=0.0, heavy=0.0, enforce=False)
+        check_case(case)
+
+
+def test_lse_in_skips_the_row_pass_and_matches():
+    cfg = si.CONFIGS["C1"].scaled(seq=640, n_q_heads=4, n_kv_heads=2, seed=9)
+    d = si.make_layer(cfg)
+    from oracle import kvmo
+    ref, lse = kvmo.scores(d["Q"], d["K"], want_lse=True)
+    p = kvm.make_params(1, 4, 2, 640, 128, torch.bfloat16)
+    ws = torch.empty(kvm.kvm_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+    out = torch.empty(1, 2, 640, device="cuda")
+    kvm.kvm_score(p, d["Q"].cuda(), d["K"].cuda(), torch.from_numpy(lse).float().cuda(), out, ws)
+    from parity import score_excess
+    assert score_excess(out.cpu().numpy(), ref) <= 1.0
+
+
+def test_c1_llama2_7b_layer_full():
+    case = _case(si.CONFIGS["C1"])
+    g = run_gpu(case)
+    check_invariants_all_units(case, g)
+    rep = check_case(case, g)
+    print("C1", rep, g.stats.units_budget_rule, g.stats.near_threshold, g.stats.min_out_len, g.stats.max_out_len)
+    assert g.stats.status == 0
+
+
+def test_compress_is_reproducible_bit_for_bit():
+    case = _case(si.CONFIGS["C1"].scaled(seq=1536, n_q_heads=4, n_kv_heads=4, seed=11))
+    a, b = run_gpu(case), run_gpu(case)
+    for f in ("c_scores", "c_out_len", "c_out_pos", "c_K_out", "c_V_out"):
+        assert np.array_equal(getattr(a, f), getattr(b, f)), f
