@@ -110,12 +110,12 @@ def run_gpu(case: Case, device="cuda") -> GpuOut:
     out_len = torch.full((B, Hkv), -7, **i32)
     stats = kvm.new_stats(device)
     kvm.kvm_segment(p, K, scores, set_id, set_start, pivot, out_len, sim, stats, ws)
-    K_out = torch.full((B, Hkv, cap, D), 777.0, dtype=Q.dtype, device=device)
-    V_out = torch.full_like(K_out, 777.0)
+    K_out = torch.full((B, Hkv, cap, D), 768.0, dtype=Q.dtype, device=device)
+    V_out = torch.full_like(K_out, 768.0)
     out_size = torch.full((B, Hkv, cap), -7, **i32)
     kvm.kvm_merge_compact(p, K, V, set_start, pivot, out_len, K_out, V_out, out_size, ws)
-    c_K = torch.full_like(K_out, 777.0)
-    c_V = torch.full_like(K_out, 777.0)
+    c_K = torch.full_like(K_out, 768.0)
+    c_V = torch.full_like(K_out, 768.0)
     c_len = torch.full((B, Hkv), -7, **i32)
     c_pos = torch.full((B, Hkv, cap), -7, **i32)
     c_scores = torch.full((B, Hkv, S), float("nan"), device=device)
@@ -259,7 +259,7 @@ def check_case(case: Case, g: Optional[GpuOut] = None, units: Optional[list] = N
         n = g_len[i]
         rep.k_err = max(rep.k_err, kv_error(g_K[i, :n], rK[i, :n]))
         rep.v_err = max(rep.v_err, kv_error(g_V[i, :n], rV[i, :n]))
-        assert (g_K[i, n:] == 777.0).all() and (g_V[i, n:] == 777.0).all(), "rows past out_len were written"
+        assert (g_K[i, n:] == 768.0).all() and (g_V[i, n:] == 768.0).all(), "rows past out_len were written"
         single = np.nonzero(np.diff(g_st[i, : n + 1]) == 1)[0]
         assert np.array_equal(g_K[i, single], K32[i, g_st[i, single]]), "singleton rows must be bit-identical"
         assert np.array_equal(g_V[i, single], V32[i, g_st[i, single]])

@@ -66,7 +66,7 @@ def test_degenerate_inputs():
     g = run_gpu(case)
     assert (g.out_len == 1).all() and (g.pivot[..., 0] == 0).all()      # all scores tie per column? pivot = arg-max
     rep = check_case(case, g)
-    np.testing.assert_allclose(g.K_out[:, :, 0], k[:, :, 0].numpy(), rtol=1e-6)
+    np.testing.assert_allclose(g.K_out[:, :, 0], k[:, :, 0].numpy(), rtol=2e-5)
     # zero keys: similarity 0 by convention, every token its own set
     K0 = torch.zeros(1, 1, 64, 64)
     case = Case(torch.randn(1, 1, 64, 64), K0, torch.randn(1, 1, 64, 64), budget=1.0, recent=0.0, heavy=0.0,
