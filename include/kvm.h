@@ -56,7 +56,8 @@ enum kvm_status {
     KVM_E_WORKSPACE = -6,   /* ws is NULL or smaller than kvm_workspace_bytes() */
     KVM_E_UNSUPPORTED = -7, /* valid request this build cannot run (e.g. non-causal) */
     KVM_E_CUDA = -8,        /* the CUDA runtime refused a launch, a copy or a driver lookup */
-    KVM_E_DEVICE_TIMEOUT = -9 /* only ever appears in kvm_stats.status: a bounded device wait gave up */
+    KVM_E_DEVICE_TIMEOUT = -9, /* only ever appears in kvm_stats.status: a bounded device wait gave up */
+    KVM_E_STATIC_LIMIT = -10 /* kvm_score_static: batch * n_q_heads * seq exceeds KVM_STATIC_SCORE_ROWS */
 };
 
 /* The paper's problem statement as a plain struct (Section 2.4; hyper-parameters of Section 5.1). */
@@ -164,6 +165,37 @@ int kvm_host_staging_bytes(const kvm_params* p, size_t* bytes);
 int kvm_compress_host(const kvm_params* p, const void* Q, const void* K, const void* V,
                       void* K_out, void* V_out, int32_t* out_len, int32_t* out_pos,
                       void* dev, size_t dev_bytes, void* cuda_stream);
+
+/*
+ * kvm_score for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a packaging variant of kvm_score, same arithmetic.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a
+ * serving engine that handed its whole memory pool to another allocator at
+ * start-up, in a plugin that is not allowed to grow the process's footprint, or
+ * on a latency path where an allocation (which may synchronise the device) is
+ * not acceptable -- and that has no spare buffer to lend as a workspace.
+ *
+ * Instead of a caller workspace, the row log-sum-exp scratch lives in a fixed
+ * array built into the library image: KVM_STATIC_SCORE_ROWS floats (4 MiB) plus
+ * 256 bytes of counters.  Every GPU that loads the library holds that array
+ * until the process exits, whether or not this function is ever called.
+ *
+ *   - Same Q, K, scores and stream arguments as kvm_score; no lse_in, no ws.
+ *   - batch * n_q_heads * seq must not exceed KVM_STATIC_SCORE_ROWS, otherwise
+ *     KVM_E_STATIC_LIMIT is returned and nothing is enqueued.
+ *   - The first call on each device looks up the array's device address (a
+ *     one-time host-side set-up, done with that device current).  Make that first
+ *     call outside any stream capture.
+ *   - All calls on one device share the one array and it keeps whatever the last
+ *     call left there.  The function re-initialises the part that must start at
+ *     zero on every call, but two calls whose kernels overlap on the GPU (different
+ *     streams, no ordering between them) race on it and give wrong scores: order
+ *     such calls on one stream or with events.
+ *   - Calls no cudaMalloc/cudaFree and no allocating library routine.
+ */
+#define KVM_STATIC_SCORE_ROWS (1 << 20)
+int kvm_score_static(const kvm_params* p, const void* Q, const void* K, float* scores, void* cuda_stream);
 
 const char* kvm_status_string(int status);
 int kvm_version(void);

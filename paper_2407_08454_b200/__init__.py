@@ -6,6 +6,6 @@
 from . import synth_inputs  # noqa: F401
 from .binding import (  # noqa: F401
     KVM_BF16, KVM_F32, Compressed, Compressor, KvmError, KvmParams, KvmStats, kvm_compress, kvm_compress_host,
-    kvm_host_staging_bytes, kvm_merge_compact, kvm_score, kvm_segment, kvm_sizes, kvm_version,
+    kvm_host_staging_bytes, kvm_merge_compact, kvm_score, kvm_score_static, kvm_segment, kvm_sizes, kvm_version,
     kvm_workspace_bytes, make_params, new_stats, read_stats, status_string,
 )

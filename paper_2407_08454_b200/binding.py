@@ -21,8 +21,9 @@ KVM_BF16, KVM_F32 = 0, 1
 KVM_OK = 0
 EXPORTS = (
     "kvm_sizes", "kvm_workspace_bytes", "kvm_score", "kvm_segment", "kvm_merge_compact", "kvm_compress",
-    "kvm_host_staging_bytes", "kvm_compress_host", "kvm_status_string", "kvm_version",
+    "kvm_host_staging_bytes", "kvm_compress_host", "kvm_score_static", "kvm_status_string", "kvm_version",
 )
+KVM_STATIC_SCORE_ROWS = 1 << 20
 
 
 class KvmParams(ctypes.Structure):
@@ -128,6 +129,13 @@ def kvm_host_staging_bytes(p: KvmParams) -> int:
 def kvm_score(p: KvmParams, Q, K, lse_in, scores, ws, stream=None) -> None:
     _check(lib().kvm_score(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(lse_in), _ptr(scores), _ptr(ws),
                            ctypes.c_size_t(ws.numel() * ws.element_size()), _stream(stream)), "kvm_score")
+
+
+def kvm_score_static(p: KvmParams, Q, K, scores, stream=None) -> None:
+    """kvm_score on the library's built-in scratch: for callers that cannot allocate a workspace.
+    batch * n_q_heads * seq must not exceed KVM_STATIC_SCORE_ROWS; calls on one device must not overlap."""
+    _check(lib().kvm_score_static(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(scores), _stream(stream)),
+           "kvm_score_static")
 
 
 def kvm_segment(p: KvmParams, K, scores, set_id, set_start, pivot, out_len, sim_out, stats, ws, stream=None) -> None:

@@ -103,6 +103,8 @@ const char* kvm_status_string(int s) {
         case KVM_E_UNSUPPORTED: return "unsupported request";
         case KVM_E_CUDA: return "CUDA runtime error";
         case KVM_E_DEVICE_TIMEOUT: return "a bounded device-side wait gave up";
+        case KVM_E_STATIC_LIMIT:
+            return "batch * n_q_heads * seq exceeds the built-in scratch of kvm_score_static (KVM_STATIC_SCORE_ROWS)";
         default: return "unknown status";
     }
 }
@@ -245,6 +247,57 @@ int kvm_compress_host(const kvm_params* p, const void* Q, const void* K, const v
     if (cudaMemcpyAsync(out_len, dL, nL, cudaMemcpyDeviceToHost, st) != cudaSuccess) return KVM_E_CUDA;
     if (cudaMemcpyAsync(out_pos, dP, nP, cudaMemcpyDeviceToHost, st) != cudaSuccess) return KVM_E_CUDA;
     return KVM_OK;
+}
+
+// ---------------------------------------------------------------------------
+// kvm_score without a caller workspace, for callers that may not allocate.
+// The scratch is part of the library image; see the declaration in kvm.h.
+namespace {
+
+constexpr int kMaxDevices = 64;
+constexpr size_t kStaticCounterBytes = 256;
+
+// [counters | row log-sum-exp].  In HOST code this name is only a stand-in for
+// the device symbol; its device address comes from cudaGetSymbolAddress below.
+static __device__ __align__(256) unsigned char g_static_score_scratch[kStaticCounterBytes +
+                                                                       (size_t)KVM_STATIC_SCORE_ROWS * sizeof(float)];
+
+void* g_static_ptr[kMaxDevices];   // device address of the array, per device; set once
+
+// One-time set-up for the current device.  Returns nullptr if the runtime refuses.
+void* static_scratch_for_current_device() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    void* ptr = __atomic_load_n(&g_static_ptr[dev], __ATOMIC_ACQUIRE);
+    if (ptr) return ptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_score_scratch) != cudaSuccess || !ptr) return nullptr;
+    __atomic_store_n(&g_static_ptr[dev], ptr, __ATOMIC_RELEASE);   // racing first calls store the same value
+    return ptr;
+}
+
+}  // namespace
+
+int kvm_score_static(const kvm_params* p, const void* Q, const void* K, float* scores, void* cuda_stream) {
+    Dims d;
+    int rc = derive(p, d);
+    if (rc != KVM_OK) return rc;
+    if (!Q || !K || !scores) return KVM_E_NULL;
+    if (misaligned(Q) || misaligned(K) || misaligned(scores)) return KVM_E_ALIGN;
+    if ((long long)d.B * d.Hq * d.S > (long long)KVM_STATIC_SCORE_ROWS) return KVM_E_STATIC_LIMIT;
+    unsigned char* base = (unsigned char*)static_scratch_for_current_device();
+    if (!base) return KVM_E_CUDA;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    // The array keeps the previous call's contents: counters must start at zero; the
+    // log-sum-exp rows are fully rewritten by the row pass before the column pass reads them.
+    if (cudaMemsetAsync(base, 0, kStaticCounterBytes, st) != cudaSuccess) return KVM_E_CUDA;
+    Workspace w;
+    w.counters = (int*)base;
+    w.lse = (float*)(base + kStaticCounterBytes);
+    w.scores = nullptr;
+    w.sim = nullptr;
+    w.set_start = nullptr;
+    w.bytes = sizeof(g_static_score_scratch);
+    return run_score(d, Q, K, nullptr, scores, w, nullptr, st) == cudaSuccess ? KVM_OK : KVM_E_CUDA;
 }
 
 }  // extern "C"
