@@ -78,7 +78,8 @@ int check_ws(const Dims& d, void* ws, size_t ws_bytes, Workspace& w) {
 
 cudaError_t run_score(const Dims& d, const void* Q, const void* K, const float* lse_in, float* scores,
                       const Workspace& w, kvm_stats* stats, cudaStream_t st) {
-    (void)stats;
+    // bf16: tensor cores (tcgen05); fp32: plain FMA, since tensor-core input rounding cannot hold the score tolerance
+    if (d.dtype == KVM_BF16) return launch_score_tc(d, Q, K, lse_in, w.lse, scores, stats, st);
     return launch_score_simt(d, Q, K, lse_in, w.lse, scores, st);
 }
 

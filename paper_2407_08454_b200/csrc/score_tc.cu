@@ -1,0 +1,485 @@
+// Aggregated attention scores on the 5th-generation tensor cores (bf16 inputs).
+//
+//   pass 1 (row pass)     lse_i = ln sum_{j<=i} exp(c q_i.k_j)                     Eq. 1, causal
+//   pass 2 (column pass)  a_j   = (1/G) sum_g sum_{i>=j} exp(c q^g_i.k_j - lse^g_i)  Algorithm 2 / Eq. 6, Section 5.2
+//
+// Both passes are the same machine.  A work item owns one 128-row "A" tile that
+// stays in shared memory (a query tile in pass 1, a key tile in pass 2) and
+// streams the 128-row "B" tiles it interacts with under the causal mask (key
+// tiles 0..it, resp. query tiles jt..T-1 of each of the G query heads).  Each
+// (A,B) pair is one 128x128xD tcgen05.mma chain into a 128-column TMEM
+// accumulator whose lanes are the A rows.  In pass 1 a thread therefore owns a
+// query row and keeps its running max / sum; in pass 2 the product is computed
+// transposed (A = keys), so a thread owns a key and adds up its column of the
+// attention map in registers, with no cross-lane reduction.
+//
+// One CTA per SM, persistent, warp-specialised:
+//   warps 0-7  epilogue: tcgen05.ld the accumulator (warp w reads TMEM lanes
+//              32*(w%4).., column half w/4), exp2 on the SFUs, row/column state
+//   warp  8    producer: TMA (cp.async.bulk.tensor, 128B swizzle) into a 4-stage ring
+//   warp  9    MMA issue: one thread issues tcgen05.mma / tcgen05.commit; owns TMEM
+// Work items are dealt in descending length, boustrophedon over the CTAs, which
+// keeps the static schedule within 2 % of a greedy one.
+//
+// Every wait on an mbarrier is bounded.  A wait that runs out raises a flag in
+// shared memory; from then on every role stops touching tensor memory and
+// barriers' payloads, finishes its loops without waiting, the outputs of the
+// affected items are poisoned with NaN, kvm_stats.status is set when given,
+// tensor memory is freed and the kernel returns.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace kvm {
+namespace {
+
+constexpr int TILE = 128;            // rows of an A or B tile = MMA M = MMA N
+constexpr int KCHUNK = 64;           // bf16 elements per 128-byte swizzle row
+constexpr int NSTAGE = 4;            // B-tile ring
+constexpr int NACC = 4;              // TMEM accumulator ring (4 x 128 columns = all 512)
+constexpr int NEPI_WARPS = 8;
+constexpr int NTHREADS = (NEPI_WARPS + 2) * 32;
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // a wait longer than 2 s is reported, not endured
+constexpr float LOG2E = 1.4426950408889634f;
+constexpr float LN2 = 0.6931471805599453f;
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false (and raises *abort_flag) if the phase never completes
+// or if another thread has already given up.
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    if (*abort_flag) return false;
+    if (mbar_try(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_try(bar, parity)) return true;
+        if ((it & 63u) == 0u) {
+            if (*abort_flag) return false;
+            if (global_ns() - t0 > WAIT_LIMIT_NS) break;
+        }
+    }
+    *abort_flag = 1;
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, uint64_t* bar, int x, int y, int z) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(ncols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 x bf16 -> fp32, one K = 16 slice.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// mbarrier arrive once all tcgen05.mma issued so far by this thread have completed.
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+// 64 consecutive fp32 columns of this thread's TMEM lane, starting at taddr.  The wait is part of the
+// same statement so that no use of the registers can be scheduled before the data has landed.
+__device__ __forceinline__ void tmem_ld64(uint32_t taddr, float* v) {
+    uint32_t r[64];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%64];\n\t"
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%65];\n\t"
+        "tcgen05.wait::ld.sync.aligned;"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
+        : "r"(taddr), "r"(taddr + 32)
+        : "memory");
+#pragma unroll
+    for (int i = 0; i < 64; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ void named_bar(int id, int nthreads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+// Shared-memory operand descriptor: K-major tile of 128-byte rows, 128-byte swizzle,
+// 8-row groups 1024 bytes apart, tile base 1024-byte aligned.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);        // start address, 16-byte units
+    d |= (uint64_t)1 << 16;                         // leading byte offset (unused with swizzle)
+    d |= (uint64_t)(1024u >> 4) << 32;              // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;                         // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;                         // 128-byte swizzle
+    return d;
+}
+// kind::f16 instruction descriptor: fp32 accumulate, bf16 A and B, both K-major, M = N = 128.
+constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TILE >> 3) << 17) | ((uint32_t)(TILE >> 4) << 24);
+
+// ------------------------------------------------------------------ static schedule
+struct Sched {
+    int P, c, NH, T, G, pass;
+    // n-th item of this CTA -> (head or unit, tile).  Items are sorted by descending length
+    // (pass 1: query tile T-1 first; pass 2: key tile 0 first) and dealt boustrophedon.
+    __device__ __forceinline__ bool item(int n, int& head, int& tile) const {
+        const long long k = (long long)n * P + ((n & 1) ? (P - 1 - c) : c);
+        if (k >= (long long)NH * T) return false;
+        const int r = (int)(k / NH);
+        head = (int)(k % NH);
+        tile = (pass == 1) ? (T - 1 - r) : r;
+        return true;
+    }
+    __device__ __forceinline__ int ntiles(int tile) const { return (pass == 1) ? tile + 1 : G * (T - tile); }
+};
+
+struct __align__(8) Barriers {
+    uint64_t full_a[2], empty_a[2];
+    uint64_t full_b[NSTAGE], empty_b[NSTAGE];
+    uint64_t acc_full[NACC], acc_empty[NACC];
+};
+
+struct alignas(16) Shared {
+    Barriers bar;
+    uint32_t tmem_base;
+    int abort_flag;
+    float part_m[2][TILE];       // cross-half partials at item end, double-buffered by item parity
+    float part_l[2][TILE];
+    alignas(16) float lse_s[2][2][64];   // [column half][tile parity][column]: pass 2 only (read as float4)
+};
+
+template <int KCH>
+__global__ void __launch_bounds__(NTHREADS, 1)
+score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                const float* __restrict__ lse_in, float* __restrict__ lse_out, float* __restrict__ scores,
+                kvm_stats* stats, int pass, int B, int Hq, int Hkv, int S, float scale2) {
+    extern __shared__ uint8_t smem_raw[];
+    constexpr uint32_t CHUNK_BYTES = TILE * 128;           // one [128 rows x 64 bf16] box
+    constexpr uint32_t TILE_BYTES = KCH * CHUNK_BYTES;
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* aligned = smem_raw + (base - smem_u32(smem_raw));
+    uint8_t* sA = aligned;                                  // 2 tiles
+    uint8_t* sB = aligned + 2 * TILE_BYTES;                 // NSTAGE tiles
+    Shared& sh = *reinterpret_cast<Shared*>(aligned + (2 + NSTAGE) * TILE_BYTES);
+    volatile int* abort_flag = &sh.abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int G = Hq / Hkv;
+    const int T = (S + TILE - 1) / TILE;
+    Sched sc{(int)gridDim.x, (int)blockIdx.x, pass == 1 ? B * Hq : B * Hkv, T, G, pass};
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < 2; ++i) { mbar_init(&sh.bar.full_a[i], 1); mbar_init(&sh.bar.empty_a[i], 1); }
+        for (int i = 0; i < NSTAGE; ++i) { mbar_init(&sh.bar.full_b[i], 1); mbar_init(&sh.bar.empty_b[i], 1); }
+        for (int i = 0; i < NACC; ++i) { mbar_init(&sh.bar.acc_full[i], 1); mbar_init(&sh.bar.acc_empty[i], NEPI_WARPS); }
+        sh.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == NEPI_WARPS + 1) tmem_alloc(&sh.tmem_base, NACC * TILE);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = sh.tmem_base;
+
+    if (warp == NEPI_WARPS) {
+        // ============================== producer ==============================
+        if (lane == 0) {
+            const CUtensorMap* mapA = (pass == 1) ? &map_q : &map_k;
+            const CUtensorMap* mapB = (pass == 1) ? &map_k : &map_q;
+            uint32_t cnt = 0;
+            bool ok = true;
+            int head, tile;
+            int last_a[2] = {-1, -1}, last_b[NSTAGE];      // parity of the last load issued per buffer (-1: none)
+            for (int s = 0; s < NSTAGE; ++s) last_b[s] = -1;
+            for (int n = 0; ok && sc.item(n, head, tile); ++n) {
+                const int ab = n & 1;
+                ok = mbar_wait(&sh.bar.empty_a[ab], ((n >> 1) & 1) ^ 1, abort_flag);
+                if (!ok) break;
+                last_a[ab] = (n >> 1) & 1;
+                mbar_expect_tx(&sh.bar.full_a[ab], TILE_BYTES);
+#pragma unroll
+                for (int kc = 0; kc < KCH; ++kc)
+                    tma_load_3d(sA + ab * TILE_BYTES + kc * CHUNK_BYTES, mapA, &sh.bar.full_a[ab], kc * KCHUNK,
+                                tile * TILE, head);
+                const int nt = sc.ntiles(tile);
+                const int b = head / (pass == 1 ? Hq : Hkv), hh = head % (pass == 1 ? Hq : Hkv);
+                const int span = T - tile;                   // pass 2: query tiles per query head
+                for (int t = 0; t < nt; ++t, ++cnt) {
+                    int bhead, btile;
+                    if (pass == 1) { bhead = b * Hkv + hh / G; btile = t; }
+                    else { bhead = b * Hq + hh * G + t / span; btile = tile + t % span; }
+                    const int s = cnt % NSTAGE;
+                    ok = mbar_wait(&sh.bar.empty_b[s], ((cnt / NSTAGE) & 1) ^ 1, abort_flag);
+                    if (!ok) break;
+                    last_b[s] = (cnt / NSTAGE) & 1;
+                    mbar_expect_tx(&sh.bar.full_b[s], TILE_BYTES);
+#pragma unroll
+                    for (int kc = 0; kc < KCH; ++kc)
+                        tma_load_3d(sB + s * TILE_BYTES + kc * CHUNK_BYTES, mapB, &sh.bar.full_b[s], kc * KCHUNK,
+                                    btile * TILE, bhead);
+                }
+            }
+            // Copies already issued complete on their own; before shared memory is given
+            // back, wait (bounded, ignoring the abort flag) for the ones nobody consumed.
+            if (*abort_flag) {
+                for (int s = 0; s < NSTAGE; ++s)
+                    for (uint32_t it = 0; last_b[s] >= 0 && it < (1u << 16); ++it)
+                        if (mbar_try(&sh.bar.full_b[s], (uint32_t)last_b[s])) break;
+                for (int s = 0; s < 2; ++s)
+                    for (uint32_t it = 0; last_a[s] >= 0 && it < (1u << 16); ++it)
+                        if (mbar_try(&sh.bar.full_a[s], (uint32_t)last_a[s])) break;
+            }
+        }
+    } else if (warp == NEPI_WARPS + 1) {
+        // ============================== MMA issue ==============================
+        if (lane == 0) {
+            uint32_t cnt = 0;
+            bool ok = true;
+            int head, tile;
+            for (int n = 0; ok && sc.item(n, head, tile); ++n) {
+                const int ab = n & 1;
+                ok = mbar_wait(&sh.bar.full_a[ab], (n >> 1) & 1, abort_flag);
+                if (!ok) break;
+                const int nt = sc.ntiles(tile);
+                for (int t = 0; t < nt; ++t, ++cnt) {
+                    const int s = cnt % NSTAGE, as = cnt % NACC;
+                    ok = mbar_wait(&sh.bar.full_b[s], (cnt / NSTAGE) & 1, abort_flag) &&
+                         mbar_wait(&sh.bar.acc_empty[as], ((cnt / NACC) & 1) ^ 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t a0 = base + ab * TILE_BYTES, b0 = base + (2 + s) * TILE_BYTES;
+                    const uint32_t d = tmem_base + as * TILE;
+#pragma unroll
+                    for (int kc = 0; kc < KCH; ++kc)
+#pragma unroll
+                        for (int ks = 0; ks < KCHUNK / 16; ++ks)
+                            umma_bf16(d, smem_desc(a0 + kc * CHUNK_BYTES + ks * 32),
+                                      smem_desc(b0 + kc * CHUNK_BYTES + ks * 32), IDESC, (kc | ks) ? 1u : 0u);
+                    umma_commit(&sh.bar.empty_b[s]);       // B stage reusable once these MMAs retire
+                    umma_commit(&sh.bar.acc_full[as]);     // accumulator ready for the epilogue
+                }
+                if (ok) umma_commit(&sh.bar.empty_a[ab]);  // A tile reusable
+            }
+        }
+    } else {
+        // ============================== epilogue ==============================
+        const int half = warp >> 2;                          // column half of every accumulator
+        const int row = (warp & 3) * 32 + lane;              // A row = TMEM lane
+        const int wg_tid = (warp & 3) * 32 + lane;           // 0..127 within the half's warpgroup
+        const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + half * 64;
+        uint32_t cnt = 0;
+        bool ok = true;
+        int head, tile;
+        for (int n = 0; sc.item(n, head, tile); ++n) {
+            const int nt = sc.ntiles(tile);
+            const int b = head / (pass == 1 ? Hq : Hkv), hh = head % (pass == 1 ? Hq : Hkv);
+            const int span = T - tile;
+            float m = -INFINITY, l = 0.f;                    // pass 1 state
+            float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;   // pass 2 state
+            for (int t = 0; t < nt; ++t, ++cnt) {
+                const int as = cnt % NACC;
+                int btile = t;
+                const float* lse_h = nullptr;
+                if (pass == 2) {
+                    btile = tile + t % span;
+                    lse_h = lse_in + ((size_t)b * Hq + hh * G + t / span) * S;
+                    // stage this tile's 64 row-lse values of our column half (log2 units; +inf past the end
+                    // of the sequence, which zeroes those columns)
+                    if (wg_tid < 64) {
+                        const int i = btile * TILE + half * 64 + wg_tid;
+                        sh.lse_s[half][cnt & 1][wg_tid] = (i < S) ? __ldg(lse_h + i) * LOG2E : INFINITY;
+                    }
+                    named_bar(1 + half, 128);
+                }
+                ok = mbar_wait(&sh.bar.acc_full[as], (cnt / NACC) & 1, abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                float v[64];
+                if (ok) {
+                    tc_fence_after();
+                    tmem_ld64(t_lane + as * TILE, v);
+                    tc_fence_before();
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh.bar.acc_empty[as]);   // values are in registers: release TMEM
+                if (!ok) continue;
+                const bool diag = (btile == tile);
+                if (pass == 1) {
+                    // valid columns of this row in this tile: c <= row on the diagonal tile, all otherwise
+                    if (diag) {
+#pragma unroll
+                        for (int c = 0; c < 64; ++c)
+                            if (half * 64 + c > row) v[c] = -INFINITY;
+                    }
+                    float mx = v[0];
+#pragma unroll
+                    for (int c = 1; c < 64; ++c) mx = fmaxf(mx, v[c]);
+                    const float mnew = fmaxf(m, mx * scale2);
+                    if (mnew > -INFINITY) {
+                        float sum0 = l * ex2(m - mnew), sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
+#pragma unroll
+                        for (int c = 0; c < 64; c += 4) {
+                            sum0 += ex2(fmaf(v[c], scale2, -mnew));
+                            sum1 += ex2(fmaf(v[c + 1], scale2, -mnew));
+                            sum2 += ex2(fmaf(v[c + 2], scale2, -mnew));
+                            sum3 += ex2(fmaf(v[c + 3], scale2, -mnew));
+                        }
+                        l = (sum0 + sum1) + (sum2 + sum3);
+                        m = mnew;
+                    }
+                } else {
+                    const float* ls = sh.lse_s[half][cnt & 1];
+                    if (diag) {
+#pragma unroll
+                        for (int c = 0; c < 64; ++c)
+                            if (half * 64 + c < row) v[c] = -INFINITY;     // query before key: masked
+                    }
+#pragma unroll
+                    for (int c = 0; c < 64; c += 4) {
+                        const float4 l4 = *reinterpret_cast<const float4*>(ls + c);
+                        acc0 += ex2(fmaf(v[c], scale2, -l4.x));
+                        acc1 += ex2(fmaf(v[c + 1], scale2, -l4.y));
+                        acc2 += ex2(fmaf(v[c + 2], scale2, -l4.z));
+                        acc3 += ex2(fmaf(v[c + 3], scale2, -l4.w));
+                    }
+                }
+            }
+            // ---- item end: combine the two column halves and store
+            const bool bad = (*abort_flag != 0);
+            const int slot = n & 1;
+            const float mine = (pass == 1) ? l : (acc0 + acc1) + (acc2 + acc3);
+            if (half == 1) { sh.part_m[slot][row] = m; sh.part_l[slot][row] = mine; }
+            named_bar(3, NEPI_WARPS * 32);
+            if (half == 0) {
+                const int gi = tile * TILE + row;
+                if (gi < S) {
+                    if (pass == 1) {
+                        const float m1 = sh.part_m[slot][row], l1 = sh.part_l[slot][row];
+                        const float M = fmaxf(m, m1);
+                        const float L = l * ex2(m - M) + l1 * ex2(m1 - M);
+                        lse_out[(size_t)head * S + gi] = bad ? NAN : (M + log2f(L)) * LN2;
+                    } else {
+                        scores[(size_t)head * S + gi] = bad ? NAN : (mine + sh.part_l[slot][row]) / (float)G;
+                    }
+                }
+            }
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0 && sh.abort_flag && stats) stats->status = KVM_E_DEVICE_TIMEOUT;
+    if (warp == NEPI_WARPS + 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, NACC * TILE);
+    }
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+// [heads, S, D] bf16, boxes of [1, 128 rows, 64 channels], 128-byte swizzle, zero fill past S.
+bool make_map(CUtensorMap* map, const void* ptr, int heads, int S, int D) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)S, (cuuint64_t)heads};
+    cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)S * D * 2};
+    cuuint32_t box[3] = {KCHUNK, TILE, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int KCH>
+cudaError_t launch_t(const Dims& d, const CUtensorMap& mq, const CUtensorMap& mk, const float* lse_in, float* lse_ws,
+                     float* scores, kvm_stats* stats, cudaStream_t st) {
+    const size_t smem = 1024 + (size_t)(2 + NSTAGE) * KCH * TILE * 128 + sizeof(Shared);
+    cudaError_t e = cudaFuncSetAttribute(score_tc_kernel<KCH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    int dev = 0, sms = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+    const int T = (d.S + TILE - 1) / TILE;
+    const float scale2 = d.scale * LOG2E;
+    const float* lse = lse_in;
+    if (!lse_in) {
+        const long long items = (long long)d.B * d.Hq * T;
+        const int grid = (int)(items < sms ? items : sms);
+        score_tc_kernel<KCH><<<grid, NTHREADS, smem, st>>>(mq, mk, nullptr, lse_ws, nullptr, stats, 1, d.B, d.Hq,
+                                                          d.Hkv, d.S, scale2);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        lse = lse_ws;
+    }
+    const long long items = (long long)d.U * T;
+    const int grid = (int)(items < sms ? items : sms);
+    score_tc_kernel<KCH><<<grid, NTHREADS, smem, st>>>(mq, mk, lse, nullptr, scores, stats, 2, d.B, d.Hq, d.Hkv, d.S,
+                                                      scale2);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_score_tc(const Dims& d, const void* Q, const void* K, const float* lse_in, float* lse_ws,
+                            float* scores, kvm_stats* stats, cudaStream_t st) {
+    CUtensorMap mq, mk;
+    if (!make_map(&mq, Q, d.B * d.Hq, d.S, d.D) || !make_map(&mk, K, d.B * d.Hkv, d.S, d.D))
+        return cudaErrorNotSupported;
+    return d.D == 128 ? launch_t<2>(d, mq, mk, lse_in, lse_ws, scores, stats, st)
+                      : launch_t<1>(d, mq, mk, lse_in, lse_ws, scores, stats, st);
+}
+
+}  // namespace kvm
