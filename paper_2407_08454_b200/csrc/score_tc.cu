@@ -14,10 +14,10 @@
 // attention map in registers, with no cross-lane reduction.
 //
 // One CTA per SM, persistent, warp-specialised:
-//   warps 0-7  epilogue: tcgen05.ld the accumulator (warp w reads TMEM lanes
-//              32*(w%4).., column half w/4), exp2 on the SFUs, row/column state
-//   warp  8    producer: TMA (cp.async.bulk.tensor, 128B swizzle) into a 4-stage ring
-//   warp  9    MMA issue: one thread issues tcgen05.mma / tcgen05.commit; owns TMEM
+//   warps 0-15 epilogue: tcgen05.ld the accumulator (warp w reads TMEM lanes
+//              32*(w%4).., column quarter w/4), exp2 on the SFUs, row/column state
+//   warp  16   producer: TMA (cp.async.bulk.tensor, 128B swizzle) into a 4-stage ring
+//   warp  17   MMA issue: one thread issues tcgen05.mma / tcgen05.commit; owns TMEM
 // Work items are dealt in descending length, boustrophedon over the CTAs, which
 // keeps the static schedule within 2 % of a greedy one.
 //
@@ -37,9 +37,10 @@ constexpr int TILE = 128;            // rows of an A or B tile = MMA M = MMA N
 constexpr int KCHUNK = 64;           // bf16 elements per 128-byte swizzle row
 constexpr int NSTAGE = 4;            // B-tile ring
 constexpr int NACC = 4;              // TMEM accumulator ring (4 x 128 columns = all 512)
-constexpr int NEPI_WARPS = 8;
+constexpr int NEPI_WARPS = 16;          // 4 TMEM lane quarters x 4 column quarters
+constexpr int QCOLS = TILE / 4;          // accumulator columns per epilogue warp
 constexpr int NTHREADS = (NEPI_WARPS + 2) * 32;
-constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // a wait longer than 2 s is reported, not endured
+constexpr long long WAIT_LIMIT_CLOCKS = 4000000000ll;   // ~2 s of SM clocks: a longer wait is reported, not endured
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float LN2 = 0.6931471805599453f;
 
@@ -68,20 +69,15 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
 }
 // Bounded wait.  Returns false (and raises *abort_flag) if the phase never completes
 // or if another thread has already given up.
-__device__ __forceinline__ unsigned long long global_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try(bar, parity)) return true;          // fast path: nothing else is touched
     if (*abort_flag) return false;
-    if (mbar_try(bar, parity)) return true;
-    const unsigned long long t0 = global_ns();
+    const long long t0 = clock64();                  // SM-local and cheap to read, unlike the global timer
     for (uint32_t it = 1;; ++it) {
         if (mbar_try(bar, parity)) return true;
         if ((it & 63u) == 0u) {
             if (*abort_flag) return false;
-            if (global_ns() - t0 > WAIT_LIMIT_NS) break;
+            if (clock64() - t0 > WAIT_LIMIT_CLOCKS) break;
         }
     }
     *abort_flag = 1;
@@ -121,19 +117,18 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                  : "memory");
 }
-// 64 consecutive fp32 columns of this thread's TMEM lane, starting at taddr.  The wait is part of the
+// 32 consecutive fp32 columns of this thread's TMEM lane, starting at taddr.  The wait is part of the
 // same statement so that no use of the registers can be scheduled before the data has landed.
-__device__ __forceinline__ void tmem_ld64(uint32_t taddr, float* v) {
-    uint32_t r[64];
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
+    uint32_t r[32];
     asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%64];\n\t"
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%65];\n\t"
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n\t"
         "tcgen05.wait::ld.sync.aligned;"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
-        : "r"(taddr), "r"(taddr + 32)
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
         : "memory");
 #pragma unroll
-    for (int i = 0; i < 64; ++i) v[i] = __uint_as_float(r[i]);
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
 __device__ __forceinline__ float ex2(float x) {
@@ -185,9 +180,9 @@ struct alignas(16) Shared {
     Barriers bar;
     uint32_t tmem_base;
     int abort_flag;
-    float part_m[2][TILE];       // cross-half partials at item end, double-buffered by item parity
-    float part_l[2][TILE];
-    alignas(16) float lse_s[2][2][64];   // [column half][tile parity][column]: pass 2 only (read as float4)
+    float part_m[2][3][TILE];    // partials of column quarters 1..3 at item end, double-buffered by item parity
+    float part_l[2][3][TILE];
+    alignas(16) float lse_s[4][2][QCOLS];   // [column quarter][tile parity][column]: pass 2 only (read as float4)
 };
 
 template <int KCH>
@@ -278,6 +273,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             uint32_t cnt = 0;
             bool ok = true;
             int head, tile;
+            const uint64_t desc_a[2] = {smem_desc(base), smem_desc(base + TILE_BYTES)};
+            const uint64_t desc_b0 = smem_desc(base + 2 * TILE_BYTES);
             for (int n = 0; ok && sc.item(n, head, tile); ++n) {
                 const int ab = n & 1;
                 ok = mbar_wait(&sh.bar.full_a[ab], (n >> 1) & 1, abort_flag);
@@ -289,14 +286,15 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                          mbar_wait(&sh.bar.acc_empty[as], ((cnt / NACC) & 1) ^ 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t a0 = base + ab * TILE_BYTES, b0 = base + (2 + s) * TILE_BYTES;
+                    // descriptors differ from the tile's first one only in the 16-byte-unit start address
+                    const uint64_t da = desc_a[ab], db = desc_b0 + (uint64_t)s * (TILE_BYTES >> 4);
                     const uint32_t d = tmem_base + as * TILE;
 #pragma unroll
                     for (int kc = 0; kc < KCH; ++kc)
 #pragma unroll
                         for (int ks = 0; ks < KCHUNK / 16; ++ks)
-                            umma_bf16(d, smem_desc(a0 + kc * CHUNK_BYTES + ks * 32),
-                                      smem_desc(b0 + kc * CHUNK_BYTES + ks * 32), IDESC, (kc | ks) ? 1u : 0u);
+                            umma_bf16(d, da + ((kc * CHUNK_BYTES + ks * 32) >> 4), db + ((kc * CHUNK_BYTES + ks * 32) >> 4),
+                                      IDESC, (kc | ks) ? 1u : 0u);
                     umma_commit(&sh.bar.empty_b[s]);       // B stage reusable once these MMAs retire
                     umma_commit(&sh.bar.acc_full[as]);     // accumulator ready for the epilogue
                 }
@@ -305,102 +303,115 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         }
     } else {
         // ============================== epilogue ==============================
-        const int half = warp >> 2;                          // column half of every accumulator
-        const int row = (warp & 3) * 32 + lane;              // A row = TMEM lane
-        const int wg_tid = (warp & 3) * 32 + lane;           // 0..127 within the half's warpgroup
-        const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + half * 64;
+        const int lq = warp & 3;                             // TMEM lane quarter this warp may read
+        const int cq = warp >> 2;                            // column quarter of every accumulator
+        const int row = lq * 32 + lane;                      // A row = TMEM lane
+        const uint32_t t_lane = tmem_base + ((uint32_t)(lq * 32) << 16) + cq * QCOLS;
         uint32_t cnt = 0;
         bool ok = true;
         int head, tile;
+        // pass 2: the row-lse of the next tile's columns is fetched one tile ahead (lane c holds column c)
+        float lse_next = 0.f;
+        auto fetch_lse = [&](int hd, int tl, int t) -> float {
+            const int b = hd / Hkv, hh = hd % Hkv, span = T - tl;
+            const int i = (tl + t % span) * TILE + cq * QCOLS + lane;
+            const float* lse_h = lse_in + ((size_t)b * Hq + hh * G + t / span) * S;
+            return (i < S) ? __ldg(lse_h + i) * LOG2E : INFINITY;   // +inf zeroes columns past the sequence end
+        };
+        if (pass == 2 && lq == 0 && sc.item(0, head, tile)) lse_next = fetch_lse(head, tile, 0);
         for (int n = 0; sc.item(n, head, tile); ++n) {
             const int nt = sc.ntiles(tile);
-            const int b = head / (pass == 1 ? Hq : Hkv), hh = head % (pass == 1 ? Hq : Hkv);
             const int span = T - tile;
+            int nhead = 0, ntile = 0;
+            const bool has_next = sc.item(n + 1, nhead, ntile);
             float m = -INFINITY, l = 0.f;                    // pass 1 state
-            float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;   // pass 2 state
+            float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};   // pass 2 state
             for (int t = 0; t < nt; ++t, ++cnt) {
                 const int as = cnt % NACC;
-                int btile = t;
-                const float* lse_h = nullptr;
+                const int btile = (pass == 1) ? t : tile + t % span;
                 if (pass == 2) {
-                    btile = tile + t % span;
-                    lse_h = lse_in + ((size_t)b * Hq + hh * G + t / span) * S;
-                    // stage this tile's 64 row-lse values of our column half (log2 units; +inf past the end
-                    // of the sequence, which zeroes those columns)
-                    if (wg_tid < 64) {
-                        const int i = btile * TILE + half * 64 + wg_tid;
-                        sh.lse_s[half][cnt & 1][wg_tid] = (i < S) ? __ldg(lse_h + i) * LOG2E : INFINITY;
+                    if (lq == 0) {
+                        sh.lse_s[cq][cnt & 1][lane] = lse_next;
+                        if (t + 1 < nt) lse_next = fetch_lse(head, tile, t + 1);
+                        else if (has_next) lse_next = fetch_lse(nhead, ntile, 0);
                     }
-                    named_bar(1 + half, 128);
+                    named_bar(1 + cq, 128);
                 }
                 ok = mbar_wait(&sh.bar.acc_full[as], (cnt / NACC) & 1, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
-                float v[64];
-                if (ok) {
+                // On the diagonal tile whole quarters are masked (skip) or fully valid (no per-element mask).
+                const bool diag = (btile == tile);
+                const bool skip = diag && ((pass == 1) ? (cq > lq) : (cq < lq));
+                const bool mask = diag && (cq == lq);
+                float v[QCOLS];
+                if (ok && !skip) {
                     tc_fence_after();
-                    tmem_ld64(t_lane + as * TILE, v);
+                    tmem_ld32(t_lane + as * TILE, v);
                     tc_fence_before();
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh.bar.acc_empty[as]);   // values are in registers: release TMEM
-                if (!ok) continue;
-                const bool diag = (btile == tile);
+                if (!ok || skip) continue;
                 if (pass == 1) {
-                    // valid columns of this row in this tile: c <= row on the diagonal tile, all otherwise
-                    if (diag) {
+                    if (mask) {
 #pragma unroll
-                        for (int c = 0; c < 64; ++c)
-                            if (half * 64 + c > row) v[c] = -INFINITY;
+                        for (int c = 0; c < QCOLS; ++c)
+                            if (c > lane) v[c] = -INFINITY;          // key after query
                     }
-                    float mx = v[0];
+                    float mx[8];
 #pragma unroll
-                    for (int c = 1; c < 64; ++c) mx = fmaxf(mx, v[c]);
-                    const float mnew = fmaxf(m, mx * scale2);
-                    if (mnew > -INFINITY) {
-                        float sum0 = l * ex2(m - mnew), sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
+                    for (int c = 0; c < 8; ++c) mx[c] = fmaxf(fmaxf(v[c], v[c + 8]), fmaxf(v[c + 16], v[c + 24]));
+                    const float mtile = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
+                                              fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
+                    const float mnew = fmaxf(m, mtile * scale2);     // finite: column 0 of a row is never masked
+                    float sum[8];
 #pragma unroll
-                        for (int c = 0; c < 64; c += 4) {
-                            sum0 += ex2(fmaf(v[c], scale2, -mnew));
-                            sum1 += ex2(fmaf(v[c + 1], scale2, -mnew));
-                            sum2 += ex2(fmaf(v[c + 2], scale2, -mnew));
-                            sum3 += ex2(fmaf(v[c + 3], scale2, -mnew));
-                        }
-                        l = (sum0 + sum1) + (sum2 + sum3);
-                        m = mnew;
-                    }
+                    for (int c = 0; c < 8; ++c) sum[c] = 0.f;
+                    sum[0] = l * ex2(m - mnew);
+#pragma unroll
+                    for (int c = 0; c < QCOLS; ++c) sum[c & 7] += ex2(fmaf(v[c], scale2, -mnew));
+                    l = ((sum[0] + sum[1]) + (sum[2] + sum[3])) + ((sum[4] + sum[5]) + (sum[6] + sum[7]));
+                    m = mnew;
                 } else {
-                    const float* ls = sh.lse_s[half][cnt & 1];
-                    if (diag) {
+                    const float* ls = sh.lse_s[cq][cnt & 1];
+                    if (mask) {
 #pragma unroll
-                        for (int c = 0; c < 64; ++c)
-                            if (half * 64 + c < row) v[c] = -INFINITY;     // query before key: masked
+                        for (int c = 0; c < QCOLS; ++c)
+                            if (c < lane) v[c] = -INFINITY;          // query before key
                     }
 #pragma unroll
-                    for (int c = 0; c < 64; c += 4) {
+                    for (int c = 0; c < QCOLS; c += 4) {
                         const float4 l4 = *reinterpret_cast<const float4*>(ls + c);
-                        acc0 += ex2(fmaf(v[c], scale2, -l4.x));
-                        acc1 += ex2(fmaf(v[c + 1], scale2, -l4.y));
-                        acc2 += ex2(fmaf(v[c + 2], scale2, -l4.z));
-                        acc3 += ex2(fmaf(v[c + 3], scale2, -l4.w));
+                        acc[c & 7] += ex2(fmaf(v[c], scale2, -l4.x));
+                        acc[(c + 1) & 7] += ex2(fmaf(v[c + 1], scale2, -l4.y));
+                        acc[(c + 2) & 7] += ex2(fmaf(v[c + 2], scale2, -l4.z));
+                        acc[(c + 3) & 7] += ex2(fmaf(v[c + 3], scale2, -l4.w));
                     }
                 }
             }
-            // ---- item end: combine the two column halves and store
+            // ---- item end: combine the four column quarters (fixed order) and store
             const bool bad = (*abort_flag != 0);
             const int slot = n & 1;
-            const float mine = (pass == 1) ? l : (acc0 + acc1) + (acc2 + acc3);
-            if (half == 1) { sh.part_m[slot][row] = m; sh.part_l[slot][row] = mine; }
-            named_bar(3, NEPI_WARPS * 32);
-            if (half == 0) {
+            const float mine = (pass == 1) ? l : ((acc[0] + acc[1]) + (acc[2] + acc[3])) + ((acc[4] + acc[5]) + (acc[6] + acc[7]));
+            if (cq > 0) { sh.part_m[slot][cq - 1][row] = m; sh.part_l[slot][cq - 1][row] = mine; }
+            named_bar(5, NEPI_WARPS * 32);
+            if (cq == 0) {
                 const int gi = tile * TILE + row;
                 if (gi < S) {
                     if (pass == 1) {
-                        const float m1 = sh.part_m[slot][row], l1 = sh.part_l[slot][row];
-                        const float M = fmaxf(m, m1);
-                        const float L = l * ex2(m - M) + l1 * ex2(m1 - M);
+                        float M = m;
+#pragma unroll
+                        for (int q = 0; q < 3; ++q) M = fmaxf(M, sh.part_m[slot][q][row]);
+                        float L = l * ex2(m - M);                    // quarter 0 always holds column 0: m finite
+#pragma unroll
+                        for (int q = 0; q < 3; ++q) {
+                            const float mq = sh.part_m[slot][q][row], lq_ = sh.part_l[slot][q][row];
+                            if (mq > -INFINITY) L += lq_ * ex2(mq - M);
+                        }
                         lse_out[(size_t)head * S + gi] = bad ? NAN : (M + log2f(L)) * LN2;
                     } else {
-                        scores[(size_t)head * S + gi] = bad ? NAN : (mine + sh.part_l[slot][row]) / (float)G;
+                        const float tot = (mine + sh.part_l[slot][0][row]) + (sh.part_l[slot][1][row] + sh.part_l[slot][2][row]);
+                        scores[(size_t)head * S + gi] = bad ? NAN : tot / (float)G;
                     }
                 }
             }
