@@ -7,8 +7,9 @@
 // stays in shared memory (a query tile in pass 1, a key tile in pass 2) and
 // streams the 128-row "B" tiles it interacts with under the causal mask (key
 // tiles 0..it, resp. query tiles jt..T-1 of each of the G query heads).  Each
-// (A,B) pair is one 128x128xD tcgen05.mma chain into a 128-column TMEM
-// accumulator whose lanes are the A rows.  In pass 1 a thread therefore owns a
+// step multiplies the A tile with two B tiles at once: a 128x256xD tcgen05.mma
+// chain (the shape at which one CTA's tensor core runs at full rate) into a
+// 256-column TMEM accumulator whose lanes are the A rows.  In pass 1 a thread therefore owns a
 // query row and keeps its running max / sum; in pass 2 the product is computed
 // transposed (A = keys), so a thread owns a key and adds up its column of the
 // attention map in registers, with no cross-lane reduction.
@@ -16,7 +17,7 @@
 // One CTA per SM, persistent, warp-specialised:
 //   warps 0-15 epilogue: tcgen05.ld the accumulator (warp w reads TMEM lanes
 //              32*(w%4).., column quarter w/4), exp2 on the SFUs, row/column state
-//   warp  16   producer: TMA (cp.async.bulk.tensor, 128B swizzle) into a 4-stage ring
+//   warp  16   producer: TMA (cp.async.bulk.tensor, 128B swizzle) into a 2-stage ring of B pairs
 //   warp  17   MMA issue: one thread issues tcgen05.mma / tcgen05.commit; owns TMEM
 // Work items are dealt in descending length, boustrophedon over the CTAs, which
 // keeps the static schedule within 2 % of a greedy one.
@@ -35,8 +36,9 @@ namespace {
 
 constexpr int TILE = 128;            // rows of an A or B tile = MMA M = MMA N
 constexpr int KCHUNK = 64;           // bf16 elements per 128-byte swizzle row
-constexpr int NSTAGE = 4;            // B-tile ring
-constexpr int NACC = 4;              // TMEM accumulator ring (4 x 128 columns = all 512)
+constexpr int NSTAGE = 2;            // ring of B pairs (two 128-row tiles each)
+constexpr int NACC = 2;              // TMEM accumulator ring (2 x 256 columns = all 512)
+constexpr int ACC_COLS = 2 * TILE;   // accumulator columns per step
 constexpr int NEPI_WARPS = 16;          // 4 TMEM lane quarters x 4 column quarters
 constexpr int QCOLS = TILE / 4;          // accumulator columns per epilogue warp
 constexpr int NTHREADS = (NEPI_WARPS + 2) * 32;
@@ -151,8 +153,11 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
     d |= (uint64_t)2 << 61;                         // 128-byte swizzle
     return d;
 }
-// kind::f16 instruction descriptor: fp32 accumulate, bf16 A and B, both K-major, M = N = 128.
-constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TILE >> 3) << 17) | ((uint32_t)(TILE >> 4) << 24);
+// kind::f16 instruction descriptor: fp32 accumulate, bf16 A and B, both K-major, M = 128, N = 128 or 256.
+constexpr uint32_t idesc_for(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(TILE >> 4) << 24);
+}
+constexpr uint32_t IDESC_N128 = idesc_for(TILE), IDESC_N256 = idesc_for(2 * TILE);
 
 // ------------------------------------------------------------------ static schedule
 struct Sched {
@@ -191,13 +196,15 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 const float* __restrict__ lse_in, float* __restrict__ lse_out, float* __restrict__ scores,
                 kvm_stats* stats, int pass, int B, int Hq, int Hkv, int S, float scale2) {
     extern __shared__ uint8_t smem_raw[];
-    constexpr uint32_t CHUNK_BYTES = TILE * 128;           // one [128 rows x 64 bf16] box
-    constexpr uint32_t TILE_BYTES = KCH * CHUNK_BYTES;
+    constexpr uint32_t CHUNK_BYTES = TILE * 128;            // one [128 rows x 64 bf16] TMA box
+    constexpr uint32_t TILE_BYTES = KCH * CHUNK_BYTES;      // an A tile: [KCH][128 rows][128 B]
+    constexpr uint32_t PAIR_CHUNK = 2 * CHUNK_BYTES;        // a B pair: [KCH][256 rows][128 B]
+    constexpr uint32_t PAIR_BYTES = KCH * PAIR_CHUNK;
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* aligned = smem_raw + (base - smem_u32(smem_raw));
-    uint8_t* sA = aligned;                                  // 2 tiles
-    uint8_t* sB = aligned + 2 * TILE_BYTES;                 // NSTAGE tiles
-    Shared& sh = *reinterpret_cast<Shared*>(aligned + (2 + NSTAGE) * TILE_BYTES);
+    uint8_t* sA = aligned;                                  // 2 A tiles
+    uint8_t* sB = aligned + 2 * TILE_BYTES;                 // NSTAGE B pairs
+    Shared& sh = *reinterpret_cast<Shared*>(aligned + 2 * TILE_BYTES + NSTAGE * PAIR_BYTES);
     volatile int* abort_flag = &sh.abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -212,12 +219,14 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         sh.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == NEPI_WARPS + 1) tmem_alloc(&sh.tmem_base, NACC * TILE);
+    if (warp == NEPI_WARPS + 1) tmem_alloc(&sh.tmem_base, NACC * ACC_COLS);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = sh.tmem_base;
 
+    // An item's B tiles are consumed two at a time ("steps"): one 128 x 256 MMA chain per step
+    // (128 x 128 for an odd last tile).  `cnt` counts steps of this CTA across items.
     if (warp == NEPI_WARPS) {
         // ============================== producer ==============================
         if (lane == 0) {
@@ -241,23 +250,26 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 const int nt = sc.ntiles(tile);
                 const int b = head / (pass == 1 ? Hq : Hkv), hh = head % (pass == 1 ? Hq : Hkv);
                 const int span = T - tile;                   // pass 2: query tiles per query head
-                for (int t = 0; t < nt; ++t, ++cnt) {
-                    int bhead, btile;
-                    if (pass == 1) { bhead = b * Hkv + hh / G; btile = t; }
-                    else { bhead = b * Hq + hh * G + t / span; btile = tile + t % span; }
+                for (int t = 0; t < nt; t += 2, ++cnt) {
                     const int s = cnt % NSTAGE;
+                    const int nh = (t + 1 < nt) ? 2 : 1;
                     ok = mbar_wait(&sh.bar.empty_b[s], ((cnt / NSTAGE) & 1) ^ 1, abort_flag);
                     if (!ok) break;
                     last_b[s] = (cnt / NSTAGE) & 1;
-                    mbar_expect_tx(&sh.bar.full_b[s], TILE_BYTES);
+                    mbar_expect_tx(&sh.bar.full_b[s], nh * TILE_BYTES);
+                    for (int h = 0; h < nh; ++h) {
+                        int bhead, btile;
+                        if (pass == 1) { bhead = b * Hkv + hh / G; btile = t + h; }
+                        else { bhead = b * Hq + hh * G + (t + h) / span; btile = tile + (t + h) % span; }
 #pragma unroll
-                    for (int kc = 0; kc < KCH; ++kc)
-                        tma_load_3d(sB + s * TILE_BYTES + kc * CHUNK_BYTES, mapB, &sh.bar.full_b[s], kc * KCHUNK,
-                                    btile * TILE, bhead);
+                        for (int kc = 0; kc < KCH; ++kc)
+                            tma_load_3d(sB + s * PAIR_BYTES + kc * PAIR_CHUNK + h * CHUNK_BYTES, mapB,
+                                        &sh.bar.full_b[s], kc * KCHUNK, btile * TILE, bhead);
+                    }
                 }
             }
             // Copies already issued complete on their own; before shared memory is given
-            // back, wait (bounded, ignoring the abort flag) for the ones nobody consumed.
+            // back, wait (bounded) for the ones nobody consumed.
             if (*abort_flag) {
                 for (int s = 0; s < NSTAGE; ++s)
                     for (uint32_t it = 0; last_b[s] >= 0 && it < (1u << 16); ++it)
@@ -273,6 +285,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             uint32_t cnt = 0;
             bool ok = true;
             int head, tile;
+            // descriptors differ from a buffer's first one only in the 16-byte-unit start address
             const uint64_t desc_a[2] = {smem_desc(base), smem_desc(base + TILE_BYTES)};
             const uint64_t desc_b0 = smem_desc(base + 2 * TILE_BYTES);
             for (int n = 0; ok && sc.item(n, head, tile); ++n) {
@@ -280,21 +293,21 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 ok = mbar_wait(&sh.bar.full_a[ab], (n >> 1) & 1, abort_flag);
                 if (!ok) break;
                 const int nt = sc.ntiles(tile);
-                for (int t = 0; t < nt; ++t, ++cnt) {
+                for (int t = 0; t < nt; t += 2, ++cnt) {
                     const int s = cnt % NSTAGE, as = cnt % NACC;
                     ok = mbar_wait(&sh.bar.full_b[s], (cnt / NSTAGE) & 1, abort_flag) &&
                          mbar_wait(&sh.bar.acc_empty[as], ((cnt / NACC) & 1) ^ 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    // descriptors differ from the tile's first one only in the 16-byte-unit start address
-                    const uint64_t da = desc_a[ab], db = desc_b0 + (uint64_t)s * (TILE_BYTES >> 4);
-                    const uint32_t d = tmem_base + as * TILE;
+                    const uint32_t idesc = (t + 1 < nt) ? IDESC_N256 : IDESC_N128;
+                    const uint64_t da = desc_a[ab], db = desc_b0 + (uint64_t)s * (PAIR_BYTES >> 4);
+                    const uint32_t d = tmem_base + as * ACC_COLS;
 #pragma unroll
                     for (int kc = 0; kc < KCH; ++kc)
 #pragma unroll
                         for (int ks = 0; ks < KCHUNK / 16; ++ks)
-                            umma_bf16(d, da + ((kc * CHUNK_BYTES + ks * 32) >> 4), db + ((kc * CHUNK_BYTES + ks * 32) >> 4),
-                                      IDESC, (kc | ks) ? 1u : 0u);
+                            umma_bf16(d, da + ((kc * CHUNK_BYTES + ks * 32) >> 4), db + ((kc * PAIR_CHUNK + ks * 32) >> 4),
+                                      idesc, (kc | ks) ? 1u : 0u);
                     umma_commit(&sh.bar.empty_b[s]);       // B stage reusable once these MMAs retire
                     umma_commit(&sh.bar.acc_full[as]);     // accumulator ready for the epilogue
                 }
@@ -304,13 +317,13 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     } else {
         // ============================== epilogue ==============================
         const int lq = warp & 3;                             // TMEM lane quarter this warp may read
-        const int cq = warp >> 2;                            // column quarter of every accumulator
+        const int cq = warp >> 2;                            // column quarter of every 128-column sub-tile
         const int row = lq * 32 + lane;                      // A row = TMEM lane
         const uint32_t t_lane = tmem_base + ((uint32_t)(lq * 32) << 16) + cq * QCOLS;
-        uint32_t cnt = 0;
+        uint32_t cnt = 0, sub = 0;                           // steps, 128-column sub-tiles
         bool ok = true;
         int head, tile;
-        // pass 2: the row-lse of the next tile's columns is fetched one tile ahead (lane c holds column c)
+        // pass 2: the row-lse of the next sub-tile's columns is fetched one sub-tile ahead (lane c holds column c)
         float lse_next = 0.f;
         auto fetch_lse = [&](int hd, int tl, int t) -> float {
             const int b = hd / Hkv, hh = hd % Hkv, span = T - tl;
@@ -326,66 +339,70 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             const bool has_next = sc.item(n + 1, nhead, ntile);
             float m = -INFINITY, l = 0.f;                    // pass 1 state
             float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};   // pass 2 state
-            for (int t = 0; t < nt; ++t, ++cnt) {
+            for (int t0 = 0; t0 < nt; t0 += 2, ++cnt) {
                 const int as = cnt % NACC;
-                const int btile = (pass == 1) ? t : tile + t % span;
-                if (pass == 2) {
-                    if (lq == 0) {
-                        sh.lse_s[cq][cnt & 1][lane] = lse_next;
-                        if (t + 1 < nt) lse_next = fetch_lse(head, tile, t + 1);
-                        else if (has_next) lse_next = fetch_lse(nhead, ntile, 0);
-                    }
-                    named_bar(1 + cq, 128);
-                }
+                const int nh = (t0 + 1 < nt) ? 2 : 1;
                 ok = mbar_wait(&sh.bar.acc_full[as], (cnt / NACC) & 1, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
-                // On the diagonal tile whole quarters are masked (skip) or fully valid (no per-element mask).
-                const bool diag = (btile == tile);
-                const bool skip = diag && ((pass == 1) ? (cq > lq) : (cq < lq));
-                const bool mask = diag && (cq == lq);
-                float v[QCOLS];
-                if (ok && !skip) {
-                    tc_fence_after();
-                    tmem_ld32(t_lane + as * TILE, v);
-                    tc_fence_before();
-                }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&sh.bar.acc_empty[as]);   // values are in registers: release TMEM
-                if (!ok || skip) continue;
-                if (pass == 1) {
-                    if (mask) {
-#pragma unroll
-                        for (int c = 0; c < QCOLS; ++c)
-                            if (c > lane) v[c] = -INFINITY;          // key after query
+                if (ok) tc_fence_after();
+                for (int h = 0; h < nh; ++h, ++sub) {
+                    const int t = t0 + h;
+                    const int btile = (pass == 1) ? t : tile + t % span;
+                    if (pass == 2) {
+                        if (lq == 0) {
+                            sh.lse_s[cq][sub & 1][lane] = lse_next;
+                            if (t + 1 < nt) lse_next = fetch_lse(head, tile, t + 1);
+                            else if (has_next) lse_next = fetch_lse(nhead, ntile, 0);
+                        }
+                        named_bar(1 + cq, 128);
                     }
-                    float mx[8];
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) mx[c] = fmaxf(fmaxf(v[c], v[c + 8]), fmaxf(v[c + 16], v[c + 24]));
-                    const float mtile = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
-                                              fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
-                    const float mnew = fmaxf(m, mtile * scale2);     // finite: column 0 of a row is never masked
-                    float sum[8];
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) sum[c] = 0.f;
-                    sum[0] = l * ex2(m - mnew);
-#pragma unroll
-                    for (int c = 0; c < QCOLS; ++c) sum[c & 7] += ex2(fmaf(v[c], scale2, -mnew));
-                    l = ((sum[0] + sum[1]) + (sum[2] + sum[3])) + ((sum[4] + sum[5]) + (sum[6] + sum[7]));
-                    m = mnew;
-                } else {
-                    const float* ls = sh.lse_s[cq][cnt & 1];
-                    if (mask) {
-#pragma unroll
-                        for (int c = 0; c < QCOLS; ++c)
-                            if (c < lane) v[c] = -INFINITY;          // query before key
+                    // On the diagonal tile whole quarters are masked (skip) or fully valid (no per-element mask).
+                    const bool diag = (btile == tile);
+                    const bool skip = diag && ((pass == 1) ? (cq > lq) : (cq < lq));
+                    const bool mask = diag && (cq == lq);
+                    float v[QCOLS];
+                    if (ok && !skip) tmem_ld32(t_lane + as * ACC_COLS + h * TILE, v);
+                    if (h == nh - 1) {                       // last read of this accumulator: release it
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&sh.bar.acc_empty[as]);
                     }
+                    if (!ok || skip) continue;
+                    if (pass == 1) {
+                        if (mask) {
 #pragma unroll
-                    for (int c = 0; c < QCOLS; c += 4) {
-                        const float4 l4 = *reinterpret_cast<const float4*>(ls + c);
-                        acc[c & 7] += ex2(fmaf(v[c], scale2, -l4.x));
-                        acc[(c + 1) & 7] += ex2(fmaf(v[c + 1], scale2, -l4.y));
-                        acc[(c + 2) & 7] += ex2(fmaf(v[c + 2], scale2, -l4.z));
-                        acc[(c + 3) & 7] += ex2(fmaf(v[c + 3], scale2, -l4.w));
+                            for (int c = 0; c < QCOLS; ++c)
+                                if (c > lane) v[c] = -INFINITY;      // key after query
+                        }
+                        float mx[8];
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) mx[c] = fmaxf(fmaxf(v[c], v[c + 8]), fmaxf(v[c + 16], v[c + 24]));
+                        const float mtile = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
+                                                  fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
+                        const float mnew = fmaxf(m, mtile * scale2); // finite: column 0 of a row is never masked
+                        float sum[8];
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) sum[c] = 0.f;
+                        sum[0] = l * ex2(m - mnew);
+#pragma unroll
+                        for (int c = 0; c < QCOLS; ++c) sum[c & 7] += ex2(fmaf(v[c], scale2, -mnew));
+                        l = ((sum[0] + sum[1]) + (sum[2] + sum[3])) + ((sum[4] + sum[5]) + (sum[6] + sum[7]));
+                        m = mnew;
+                    } else {
+                        const float* ls = sh.lse_s[cq][sub & 1];
+                        if (mask) {
+#pragma unroll
+                            for (int c = 0; c < QCOLS; ++c)
+                                if (c < lane) v[c] = -INFINITY;      // query before key
+                        }
+#pragma unroll
+                        for (int c = 0; c < QCOLS; c += 4) {
+                            const float4 l4 = *reinterpret_cast<const float4*>(ls + c);
+                            acc[c & 7] += ex2(fmaf(v[c], scale2, -l4.x));
+                            acc[(c + 1) & 7] += ex2(fmaf(v[c + 1], scale2, -l4.y));
+                            acc[(c + 2) & 7] += ex2(fmaf(v[c + 2], scale2, -l4.z));
+                            acc[(c + 3) & 7] += ex2(fmaf(v[c + 3], scale2, -l4.w));
+                        }
                     }
                 }
             }
@@ -421,7 +438,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     if (threadIdx.x == 0 && sh.abort_flag && stats) stats->status = KVM_E_DEVICE_TIMEOUT;
     if (warp == NEPI_WARPS + 1) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, NACC * TILE);
+        tmem_dealloc(tmem_base, NACC * ACC_COLS);
     }
 }
 
@@ -458,7 +475,7 @@ bool make_map(CUtensorMap* map, const void* ptr, int heads, int S, int D) {
 template <int KCH>
 cudaError_t launch_t(const Dims& d, const CUtensorMap& mq, const CUtensorMap& mk, const float* lse_in, float* lse_ws,
                      float* scores, kvm_stats* stats, cudaStream_t st) {
-    const size_t smem = 1024 + (size_t)(2 + NSTAGE) * KCH * TILE * 128 + sizeof(Shared);
+    const size_t smem = 1024 + (size_t)(2 + 2 * NSTAGE) * KCH * TILE * 128 + sizeof(Shared);
     cudaError_t e = cudaFuncSetAttribute(score_tc_kernel<KCH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     int dev = 0, sms = 0;
