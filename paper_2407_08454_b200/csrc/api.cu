@@ -50,6 +50,8 @@ struct Workspace {
     float* scores;      // [U,S]
     float* sim;         // [U,S]
     int32_t* set_start; // [U,cap+1]
+    int32_t* set_id;    // [U,S]
+    float* merge_part;  // partial sums of sets that cross token tiles
     size_t bytes;
 };
 
@@ -62,6 +64,8 @@ Workspace carve(const Dims& d, void* base) {
     w.scores = (float*)take((size_t)d.U * d.S * sizeof(float));
     w.sim = (float*)take((size_t)d.U * d.S * sizeof(float));
     w.set_start = (int32_t*)take((size_t)d.U * (d.cap + 1) * sizeof(int32_t));
+    w.set_id = (int32_t*)take((size_t)d.U * d.S * sizeof(int32_t));
+    w.merge_part = (float*)take(merge_scratch_floats(d) * sizeof(float));
     w.bytes = off;
     return w;
 }
@@ -170,8 +174,9 @@ int kvm_merge_compact(const kvm_params* p, const void* K, const void* V, const i
     if (misaligned(K) || misaligned(V) || misaligned(K_out) || misaligned(V_out)) return KVM_E_ALIGN;
     Workspace w;
     if ((rc = check_ws(d, ws, ws_bytes, w)) != KVM_OK) return rc;
-    return launch_merge(d, K, V, set_start, pivot, out_len, K_out, V_out, out_size, (cudaStream_t)cuda_stream) ==
-                   cudaSuccess
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (launch_token_sets(d, set_start, out_len, w.set_id, st) != cudaSuccess) return KVM_E_CUDA;
+    return launch_merge(d, K, V, set_start, pivot, w.set_id, K_out, V_out, out_size, w.merge_part, st) == cudaSuccess
                ? KVM_OK
                : KVM_E_CUDA;
 }
@@ -192,9 +197,9 @@ int kvm_compress(const kvm_params* p, const void* Q, const void* K, const void* 
     float* scores = scores_out ? scores_out : w.scores;
     if (run_score(d, Q, K, nullptr, scores, w, stats, st) != cudaSuccess) return KVM_E_CUDA;
     if (launch_similarity(d, K, w.sim, st) != cudaSuccess) return KVM_E_CUDA;
-    if (launch_segment(d, scores, w.sim, nullptr, w.set_start, out_pos, out_len, stats, st) != cudaSuccess)
+    if (launch_segment(d, scores, w.sim, w.set_id, w.set_start, out_pos, out_len, stats, st) != cudaSuccess)
         return KVM_E_CUDA;
-    if (launch_merge(d, K, V, w.set_start, out_pos, out_len, K_out, V_out, nullptr, st) != cudaSuccess)
+    if (launch_merge(d, K, V, w.set_start, out_pos, w.set_id, K_out, V_out, nullptr, w.merge_part, st) != cudaSuccess)
         return KVM_E_CUDA;
     return KVM_OK;
 }
@@ -297,6 +302,8 @@ int kvm_score_static(const kvm_params* p, const void* Q, const void* K, float* s
     w.scores = nullptr;
     w.sim = nullptr;
     w.set_start = nullptr;
+    w.set_id = nullptr;
+    w.merge_part = nullptr;
     w.bytes = sizeof(g_static_score_scratch);
     return run_score(d, Q, K, nullptr, scores, w, nullptr, st) == cudaSuccess ? KVM_OK : KVM_E_CUDA;
 }

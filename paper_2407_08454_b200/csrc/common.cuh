@@ -57,8 +57,11 @@ cudaError_t launch_score_tc(const Dims& d, const void* Q, const void* K, const f
 cudaError_t launch_similarity(const Dims& d, const void* K, float* sim, cudaStream_t st);
 cudaError_t launch_segment(const Dims& d, const float* scores, const float* sim, int32_t* set_id,
                            int32_t* set_start, int32_t* pivot, int32_t* out_len, kvm_stats* stats, cudaStream_t st);
+size_t merge_scratch_floats(const Dims& d);
+cudaError_t launch_token_sets(const Dims& d, const int32_t* set_start, const int32_t* out_len, int32_t* set_id,
+                              cudaStream_t st);
 cudaError_t launch_merge(const Dims& d, const void* K, const void* V, const int32_t* set_start,
-                         const int32_t* pivot, const int32_t* out_len, void* K_out, void* V_out,
-                         int32_t* out_size, cudaStream_t st);
+                         const int32_t* pivot, const int32_t* set_id, void* K_out, void* V_out, int32_t* out_size,
+                         float* scratch, cudaStream_t st);
 
 }  // namespace kvm

@@ -3,10 +3,20 @@
 // Algorithm 2):
 //   g_j = exp(-|k_p - k_j|^2 / (2 sigma^2)),  K* = sum g_j k_j / sum g_j,
 //   V* = n * sum g_j v_j / sum g_j.
-// Bandwidth-bound: K and V are each read once with 16-byte loads (the pivot
-// row is read a second time, from cache).  A group of LPR lanes owns one output
-// row and walks its set; fp32 accumulation; one round-to-nearest-even
-// conversion at the store.  Sets of one token are copied bit for bit.
+//
+// Bandwidth-bound, and sets can be arbitrarily long, so the work is split by
+// TOKENS, not by sets: a block owns TOK consecutive tokens of one unit, pulls
+// their K and V rows into shared memory with two bulk copies, and
+//   phase 1  one lane group per token computes its weight g_j (the pivot row is
+//            taken from shared memory when it lies in the tile, else from L2);
+//   phase 2  one thread per (tensor, channel) walks the tile's tokens in order,
+//            adding g_j x_j, and flushes at every set boundary.
+// A set that lies inside the tile is finished there.  A set that crosses tile
+// boundaries leaves fp32 partial sums in a scratch slot per (unit, tile): "head"
+// = the tile's tokens before its first boundary, "tail" = after its last; a small
+// second kernel adds a crossing set's slots in tile order and stores the row.
+// Nothing uses atomics: every sum has a fixed order, results are reproducible.
+// Sets of one token are copied bit for bit.
 #include "common.cuh"
 
 namespace kvm {
@@ -14,110 +24,239 @@ namespace {
 
 constexpr float LOG2E = 1.4426950408889634f;
 
-template <typename T, int D>
-__global__ void __launch_bounds__(256) merge_compact_kernel(const T* __restrict__ K, const T* __restrict__ V,
-                                                            const int32_t* __restrict__ set_start,
-                                                            const int32_t* __restrict__ pivot,
-                                                            const int32_t* __restrict__ out_len,
-                                                            T* __restrict__ K_out, T* __restrict__ V_out,
-                                                            int32_t* __restrict__ out_size, int S, int cap,
-                                                            long long n_rows, float neg_inv_2s2_log2e, int scale_v) {
-    constexpr int N = Vec<T>::N;
-    constexpr int LPR = D / N;
-    const long long row = ((long long)blockIdx.x * blockDim.x + threadIdx.x) / LPR;   // u*cap + s
-    if (row >= n_rows) return;
-    const int lane = threadIdx.x % LPR;
-    const unsigned gmask = (LPR == 32) ? 0xffffffffu : (((1u << LPR) - 1u) << ((threadIdx.x % 32) / LPR * LPR));
-    const long long u = row / cap;
-    const int s = (int)(row % cap);
-    if (s >= out_len[u]) return;
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+template <typename T> __device__ __forceinline__ float elem_to_f32(T v);
+template <> __device__ __forceinline__ float elem_to_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ float elem_to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T f32_to_elem(float v);
+template <> __device__ __forceinline__ float f32_to_elem<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 f32_to_elem<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// set_id[u][j] = index of the set holding token j, from the sets' start positions.
+__global__ void __launch_bounds__(256) token_set_kernel(const int32_t* __restrict__ set_start,
+                                                        const int32_t* __restrict__ out_len,
+                                                        int32_t* __restrict__ set_id, int S, int cap) {
+    const int u = blockIdx.y;
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= S) return;
     const int32_t* st = set_start + (size_t)u * (cap + 1);
-    const int lo = st[s], hi = st[s + 1];
-    const int n = hi - lo;
-    const T* Ku = K + (size_t)u * S * D + lane * N;
-    const T* Vu = V + (size_t)u * S * D + lane * N;
-    T* ko = K_out + (size_t)row * D + lane * N;
-    T* vo = V_out + (size_t)row * D + lane * N;
-    if (lane == 0 && out_size) out_size[row] = n;
-
-    if (n == 1) {
-        *reinterpret_cast<uint4*>(ko) = ldg16(Ku + (size_t)lo * D);
-        *reinterpret_cast<uint4*>(vo) = ldg16(Vu + (size_t)lo * D);
-        return;
+    int lo = 0, hi = min(out_len[u], cap);      // largest s in [0, hi) with st[s] <= j
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (__ldg(st + mid) <= j) lo = mid; else hi = mid;
     }
-    const int p = pivot[row];
-    float kp[N];
-    Vec<T>::unpack(ldg16(Ku + (size_t)p * D), kp);
-    float accK[N], accV[N], gsum = 0.f;
-#pragma unroll
-    for (int e = 0; e < N; ++e) { accK[e] = 0.f; accV[e] = 0.f; }
-
-    for (int jb = lo; jb < hi; jb += 2) {
-        const bool two = (jb + 1 < hi);
-        const uint4 rk0 = ldg16(Ku + (size_t)jb * D);
-        const uint4 rv0 = ldg16(Vu + (size_t)jb * D);
-        const uint4 rk1 = two ? ldg16(Ku + (size_t)(jb + 1) * D) : make_uint4(0, 0, 0, 0);
-        const uint4 rv1 = two ? ldg16(Vu + (size_t)(jb + 1) * D) : make_uint4(0, 0, 0, 0);
-        float k0[N], v0[N], k1[N], v1[N];
-        Vec<T>::unpack(rk0, k0); Vec<T>::unpack(rv0, v0);
-        Vec<T>::unpack(rk1, k1); Vec<T>::unpack(rv1, v1);
-        float d0 = 0.f, d1 = 0.f;
-#pragma unroll
-        for (int e = 0; e < N; ++e) {
-            const float a = kp[e] - k0[e], b = kp[e] - k1[e];
-            d0 = fmaf(a, a, d0);
-            d1 = fmaf(b, b, d1);
-        }
-#pragma unroll
-        for (int off = 1; off < LPR; off <<= 1) {
-            d0 += __shfl_xor_sync(gmask, d0, off);
-            d1 += __shfl_xor_sync(gmask, d1, off);
-        }
-        const float g0 = exp2f(d0 * neg_inv_2s2_log2e);
-        const float g1 = two ? exp2f(d1 * neg_inv_2s2_log2e) : 0.f;
-        gsum += g0 + g1;
-#pragma unroll
-        for (int e = 0; e < N; ++e) {
-            accK[e] = fmaf(g0, k0[e], accK[e]);
-            accV[e] = fmaf(g0, v0[e], accV[e]);
-            accK[e] = fmaf(g1, k1[e], accK[e]);
-            accV[e] = fmaf(g1, v1[e], accV[e]);
-        }
-    }
-    const float inv = 1.f / gsum;                       // gsum >= 1: the pivot's own weight is exp(0)
-    const float vmul = scale_v ? (float)n * inv : inv;
-#pragma unroll
-    for (int e = 0; e < N; ++e) { accK[e] *= inv; accV[e] *= vmul; }
-    *reinterpret_cast<uint4*>(ko) = Vec<T>::pack(accK);
-    *reinterpret_cast<uint4*>(vo) = Vec<T>::pack(accV);
+    set_id[(size_t)u * S + j] = lo;
 }
 
-template <typename T, int D>
+// Scratch layout per (unit, tile): [head | tail] x (2*D sums: K channels then V channels), and 2 weight sums.
+template <int D> struct Slots {
+    float* sums;      // [U][T][2][2*D]
+    float* gsum;      // [U][T][2]
+    __device__ __forceinline__ float* s(long long u, int T, int tile, int which) const {
+        return sums + (((size_t)u * T + tile) * 2 + which) * (2 * D);
+    }
+    __device__ __forceinline__ float* g(long long u, int T, int tile, int which) const {
+        return gsum + ((size_t)u * T + tile) * 2 + which;
+    }
+};
+
+template <typename T, int D, int TOK>
+__global__ void __launch_bounds__(2 * D) merge_tile_kernel(const T* __restrict__ K, const T* __restrict__ V,
+                                                           const int32_t* __restrict__ set_start,
+                                                           const int32_t* __restrict__ pivot,
+                                                           const int32_t* __restrict__ set_id,
+                                                           T* __restrict__ K_out, T* __restrict__ V_out,
+                                                           int32_t* __restrict__ out_size, Slots<D> slots, int S,
+                                                           int cap, float neg_inv_2s2_log2e, int scale_v) {
+    constexpr int N = Vec<T>::N;          // elements per 16 bytes
+    constexpr int LPR = D / N;            // lanes per row
+    constexpr int NT = 2 * D;             // threads: one per (tensor, channel)
+    constexpr int NWORK = NT / LPR;       // lane groups in phase 1
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    T* sK = reinterpret_cast<T*>(smem_raw);
+    T* sV = sK + TOK * D;
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int s_sid[TOK], s_piv[TOK], s_beg[TOK], s_end[TOK];
+    __shared__ float s_g[TOK];
+
+    const int tile = blockIdx.x, Tn = gridDim.x;
+    const long long u = blockIdx.y;
+    const int tok0 = tile * TOK;
+    const int ntok = min(TOK, S - tok0);
+    const T* Ku = K + (size_t)u * S * D;
+    const T* Vu = V + (size_t)u * S * D;
+    const int32_t* st = set_start + (size_t)u * (cap + 1);
+    const uint32_t bytes = (uint32_t)ntok * D * sizeof(T);
+
+    if (threadIdx.x == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&bar)));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(&bar)), "r"(2 * bytes)
+                     : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(smem_u32(sK)), "l"(Ku + (size_t)tok0 * D), "r"(bytes), "r"(smem_u32(&bar)) : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(smem_u32(sV)), "l"(Vu + (size_t)tok0 * D), "r"(bytes), "r"(smem_u32(&bar)) : "memory");
+    }
+    // per-token set data while the rows are in flight
+    for (int j = threadIdx.x; j < ntok; j += NT) {
+        const int sid = __ldg(set_id + (size_t)u * S + tok0 + j);
+        s_sid[j] = sid;
+        s_piv[j] = __ldg(pivot + (size_t)u * cap + sid);
+        s_beg[j] = __ldg(st + sid);
+        s_end[j] = __ldg(st + sid + 1);
+    }
+    __syncthreads();                     // barrier initialised + metadata visible
+    {
+        // The copies were issued by this block and always complete; the wait is still bounded.
+        uint32_t done = 0;
+        for (uint32_t it = 0; it < (1u << 26) && !done; ++it)
+            asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n\t"
+                         "selp.u32 %0, 1, 0, p;\n\t}" : "=r"(done) : "r"(smem_u32(&bar)) : "memory");
+    }
+
+    // ---- phase 1: weights
+    {
+        const int w = threadIdx.x / LPR, lane = threadIdx.x % LPR;
+        const unsigned gmask = (LPR == 32) ? 0xffffffffu : (((1u << LPR) - 1u) << ((threadIdx.x % 32) / LPR * LPR));
+        for (int j = w; j < ntok; j += NWORK) {
+            const int p = s_piv[j];
+            float kj[N], kp[N];
+            Vec<T>::unpack(*reinterpret_cast<const uint4*>(sK + (size_t)j * D + lane * N), kj);
+            if (p >= tok0 && p < tok0 + ntok)
+                Vec<T>::unpack(*reinterpret_cast<const uint4*>(sK + (size_t)(p - tok0) * D + lane * N), kp);
+            else
+                Vec<T>::unpack(ldg16(Ku + (size_t)p * D + lane * N), kp);
+            float d2 = 0.f;
+#pragma unroll
+            for (int e = 0; e < N; ++e) { const float a = kp[e] - kj[e]; d2 = fmaf(a, a, d2); }
+#pragma unroll
+            for (int off = 1; off < LPR; off <<= 1) d2 += __shfl_xor_sync(gmask, d2, off);
+            if (lane == 0) s_g[j] = exp2f(d2 * neg_inv_2s2_log2e);
+        }
+    }
+    __syncthreads();
+
+    // ---- phase 2: one thread per (tensor, channel) walks the tokens
+    const int which = threadIdx.x / D, ch = threadIdx.x % D;     // 0: K, 1: V
+    const T* sX = which ? sV : sK;
+    T* out = which ? V_out : K_out;
+    const int tile_end = tok0 + ntok;
+    float acc = 0.f, gs = 0.f;
+    T first_raw = sX[ch];
+    auto flush = [&](int j_last) {       // the set whose last token in this tile is j_last
+        const int sid = s_sid[j_last], beg = s_beg[j_last], end = s_end[j_last];
+        const bool started_here = beg >= tok0, closes_here = end <= tile_end;
+        if (started_here && closes_here) {
+            const int n = end - beg;
+            T r;
+            if (n == 1) r = first_raw;
+            else r = f32_to_elem<T>(which && scale_v ? acc * ((float)n / gs) : acc / gs);
+            out[((size_t)u * cap + sid) * D + ch] = r;
+            if (out_size && threadIdx.x == 0) out_size[(size_t)u * cap + sid] = n;
+        } else {
+            const int slot = started_here ? 1 : 0;               // tail : head
+            slots.s(u, Tn, tile, slot)[threadIdx.x] = acc;
+            if (threadIdx.x == 0) *slots.g(u, Tn, tile, slot) = gs;
+        }
+    };
+    for (int j = 0; j < ntok; ++j) {
+        if (j > 0 && s_sid[j] != s_sid[j - 1]) {
+            flush(j - 1);
+            acc = 0.f; gs = 0.f;
+            first_raw = sX[(size_t)j * D + ch];
+        }
+        const float g = s_g[j];
+        acc = fmaf(g, elem_to_f32<T>(sX[(size_t)j * D + ch]), acc);
+        gs += g;
+    }
+    flush(ntok - 1);
+}
+
+// Sets that cross a tile boundary: the block of the LAST boundary a set crosses adds its slots in tile order.
+template <typename T, int D, int TOK>
+__global__ void __launch_bounds__(2 * D) merge_fixup_kernel(const int32_t* __restrict__ set_start,
+                                                            const int32_t* __restrict__ set_id,
+                                                            T* __restrict__ K_out, T* __restrict__ V_out,
+                                                            int32_t* __restrict__ out_size, Slots<D> slots, int S,
+                                                            int cap, int Tn, int scale_v) {
+    const int c = blockIdx.x + 1;                 // boundary between tiles c-1 and c
+    const long long u = blockIdx.y;
+    const int b = c * TOK;
+    if (b >= S) return;
+    const int32_t* sid_u = set_id + (size_t)u * S;
+    const int sid = sid_u[b];
+    if (sid_u[b - 1] != sid) return;              // no set crosses here
+    const int32_t* st = set_start + (size_t)u * (cap + 1);
+    const int beg = st[sid], end = st[sid + 1];
+    if (end > b + TOK) return;                    // crosses a later boundary too: finished there
+    const int c_first = beg / TOK;                // tile holding the set's first token (its tail slot)
+    float acc = slots.s(u, Tn, c_first, 1)[threadIdx.x];
+    float gs = *slots.g(u, Tn, c_first, 1);
+    for (int t = c_first + 1; t <= c; ++t) {
+        acc += slots.s(u, Tn, t, 0)[threadIdx.x];
+        gs += *slots.g(u, Tn, t, 0);
+    }
+    const int which = threadIdx.x / D, ch = threadIdx.x % D;
+    const int n = end - beg;
+    T* out = which ? V_out : K_out;
+    out[((size_t)u * cap + sid) * D + ch] = f32_to_elem<T>(which && scale_v ? acc * ((float)n / gs) : acc / gs);
+    if (out_size && threadIdx.x == 0) out_size[(size_t)u * cap + sid] = n;
+}
+
+template <typename T, int D, int TOK>
 cudaError_t launch_t(const Dims& d, const void* K, const void* V, const int32_t* set_start, const int32_t* pivot,
-                     const int32_t* out_len, void* K_out, void* V_out, int32_t* out_size, cudaStream_t st) {
-    constexpr int LPR = D / Vec<T>::N;
-    const long long rows = (long long)d.U * d.cap;
-    const long long threads = rows * LPR;
-    const unsigned blocks = (unsigned)((threads + 255) / 256);
+                     const int32_t* set_id, void* K_out, void* V_out, int32_t* out_size, float* scratch,
+                     cudaStream_t st) {
+    const int Tn = (d.S + TOK - 1) / TOK;
+    Slots<D> slots;
+    slots.sums = scratch;
+    slots.gsum = scratch + (size_t)d.U * Tn * 2 * (2 * D);
+    const size_t smem = (size_t)2 * TOK * D * sizeof(T);
+    cudaError_t e = cudaFuncSetAttribute(merge_tile_kernel<T, D, TOK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)smem);
+    if (e != cudaSuccess) return e;
     const float c = -LOG2E / (2.f * d.sigma * d.sigma);
-    merge_compact_kernel<T, D><<<blocks, 256, 0, st>>>((const T*)K, (const T*)V, set_start, pivot, out_len,
-                                                       (T*)K_out, (T*)V_out, out_size, d.S, d.cap, rows, c,
-                                                       d.scale_v);
-    return cudaGetLastError();
+    merge_tile_kernel<T, D, TOK><<<dim3(Tn, d.U), 2 * D, smem, st>>>(
+        (const T*)K, (const T*)V, set_start, pivot, set_id, (T*)K_out, (T*)V_out, out_size, slots, d.S, d.cap, c,
+        d.scale_v);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    if (Tn > 1) {
+        merge_fixup_kernel<T, D, TOK><<<dim3(Tn - 1, d.U), 2 * D, 0, st>>>(set_start, set_id, (T*)K_out, (T*)V_out,
+                                                                          out_size, slots, d.S, d.cap, Tn, d.scale_v);
+        e = cudaGetLastError();
+    }
+    return e;
 }
 
 }  // namespace
 
+// Tokens per tile: 128 for 2-byte elements, 64 for 4-byte ones (64 KB resp. 32-64 KB of shared memory).
+size_t merge_scratch_floats(const Dims& d) {
+    const int TOK = d.dtype == KVM_BF16 ? 128 : 64;
+    const size_t Tn = (d.S + TOK - 1) / TOK;
+    return (size_t)d.U * Tn * 2 * (2 * d.D) + (size_t)d.U * Tn * 2;
+}
+
+cudaError_t launch_token_sets(const Dims& d, const int32_t* set_start, const int32_t* out_len, int32_t* set_id,
+                              cudaStream_t st) {
+    token_set_kernel<<<dim3((d.S + 255) / 256, d.U), 256, 0, st>>>(set_start, out_len, set_id, d.S, d.cap);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_merge(const Dims& d, const void* K, const void* V, const int32_t* set_start,
-                         const int32_t* pivot, const int32_t* out_len, void* K_out, void* V_out,
-                         int32_t* out_size, cudaStream_t st) {
+                         const int32_t* pivot, const int32_t* set_id, void* K_out, void* V_out, int32_t* out_size,
+                         float* scratch, cudaStream_t st) {
     if (d.dtype == KVM_BF16) {
-        return d.D == 128
-                   ? launch_t<__nv_bfloat16, 128>(d, K, V, set_start, pivot, out_len, K_out, V_out, out_size, st)
-                   : launch_t<__nv_bfloat16, 64>(d, K, V, set_start, pivot, out_len, K_out, V_out, out_size, st);
+        return d.D == 128 ? launch_t<__nv_bfloat16, 128, 128>(d, K, V, set_start, pivot, set_id, K_out, V_out,
+                                                              out_size, scratch, st)
+                          : launch_t<__nv_bfloat16, 64, 128>(d, K, V, set_start, pivot, set_id, K_out, V_out,
+                                                             out_size, scratch, st);
     }
-    return d.D == 128 ? launch_t<float, 128>(d, K, V, set_start, pivot, out_len, K_out, V_out, out_size, st)
-                      : launch_t<float, 64>(d, K, V, set_start, pivot, out_len, K_out, V_out, out_size, st);
+    return d.D == 128
+               ? launch_t<float, 128, 64>(d, K, V, set_start, pivot, set_id, K_out, V_out, out_size, scratch, st)
+               : launch_t<float, 64, 64>(d, K, V, set_start, pivot, set_id, K_out, V_out, out_size, scratch, st);
 }
 
 }  // namespace kvm
