@@ -138,6 +138,35 @@ __device__ __forceinline__ float ex2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+// Packed pairs of fp32 (one issue slot for two lanes of work on this architecture).
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t p, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(p));
+}
+__device__ __forceinline__ uint64_t ffma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ uint64_t fadd2(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+__device__ __forceinline__ float hsum2(uint64_t p) {
+    float lo, hi;
+    unpack2(p, lo, hi);
+    return lo + hi;
+}
 __device__ __forceinline__ void named_bar(int id, int nthreads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
@@ -187,7 +216,8 @@ struct alignas(16) Shared {
     int abort_flag;
     float part_m[2][3][TILE];    // partials of column quarters 1..3 at item end, double-buffered by item parity
     float part_l[2][3][TILE];
-    alignas(16) float lse_s[4][2][QCOLS];   // [column quarter][tile parity][column]: pass 2 only (read as float4)
+    alignas(16) float nlse_s[NEPI_WARPS][2][QCOLS];   // pass 2: each warp's own copy of -lse*log2(e) of its 32
+                                                      // columns, double-buffered by sub-tile parity
 };
 
 template <int KCH>
@@ -323,22 +353,24 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         uint32_t cnt = 0, sub = 0;                           // steps, 128-column sub-tiles
         bool ok = true;
         int head, tile;
-        // pass 2: the row-lse of the next sub-tile's columns is fetched one sub-tile ahead (lane c holds column c)
+        // pass 2: -lse*log2(e) of the next sub-tile's columns is fetched one sub-tile ahead (lane c holds
+        // column c); every warp keeps its own staged copy, so no barrier is needed to share it
         float lse_next = 0.f;
         auto fetch_lse = [&](int hd, int tl, int t) -> float {
             const int b = hd / Hkv, hh = hd % Hkv, span = T - tl;
             const int i = (tl + t % span) * TILE + cq * QCOLS + lane;
             const float* lse_h = lse_in + ((size_t)b * Hq + hh * G + t / span) * S;
-            return (i < S) ? __ldg(lse_h + i) * LOG2E : INFINITY;   // +inf zeroes columns past the sequence end
+            return (i < S) ? __ldg(lse_h + i) * -LOG2E : -INFINITY;   // -inf zeroes columns past the sequence end
         };
-        if (pass == 2 && lq == 0 && sc.item(0, head, tile)) lse_next = fetch_lse(head, tile, 0);
+        if (pass == 2 && sc.item(0, head, tile)) lse_next = fetch_lse(head, tile, 0);
+        const uint64_t sc2 = pack2(scale2, scale2);
         for (int n = 0; sc.item(n, head, tile); ++n) {
             const int nt = sc.ntiles(tile);
             const int span = T - tile;
             int nhead = 0, ntile = 0;
             const bool has_next = sc.item(n + 1, nhead, ntile);
             float m = -INFINITY, l = 0.f;                    // pass 1 state
-            float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};   // pass 2 state
+            uint64_t acc2[4] = {0ull, 0ull, 0ull, 0ull};     // pass 2 state: four packed pairs of partial sums
             for (int t0 = 0; t0 < nt; t0 += 2, ++cnt) {
                 const int as = cnt % NACC;
                 const int nh = (t0 + 1 < nt) ? 2 : 1;
@@ -349,12 +381,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     const int t = t0 + h;
                     const int btile = (pass == 1) ? t : tile + t % span;
                     if (pass == 2) {
-                        if (lq == 0) {
-                            sh.lse_s[cq][sub & 1][lane] = lse_next;
-                            if (t + 1 < nt) lse_next = fetch_lse(head, tile, t + 1);
-                            else if (has_next) lse_next = fetch_lse(nhead, ntile, 0);
-                        }
-                        named_bar(1 + cq, 128);
+                        sh.nlse_s[warp][sub & 1][lane] = lse_next;
+                        if (t + 1 < nt) lse_next = fetch_lse(head, tile, t + 1);
+                        else if (has_next) lse_next = fetch_lse(nhead, ntile, 0);
+                        __syncwarp();
                     }
                     // On the diagonal tile whole quarters are masked (skip) or fully valid (no per-element mask).
                     const bool diag = (btile == tile);
@@ -374,22 +404,28 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                             for (int c = 0; c < QCOLS; ++c)
                                 if (c > lane) v[c] = -INFINITY;      // key after query
                         }
-                        float mx[8];
+                        float mx[4];
 #pragma unroll
-                        for (int c = 0; c < 8; ++c) mx[c] = fmaxf(fmaxf(v[c], v[c + 8]), fmaxf(v[c + 16], v[c + 24]));
-                        const float mtile = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
-                                                  fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
+                        for (int c = 0; c < 4; ++c) {
+                            mx[c] = fmax3(v[c], v[c + 4], v[c + 8]);
+                            mx[c] = fmax3(mx[c], v[c + 12], v[c + 16]);
+                            mx[c] = fmax3(mx[c], v[c + 20], v[c + 24]);
+                            mx[c] = fmaxf(mx[c], v[c + 28]);
+                        }
+                        const float mtile = fmaxf(fmax3(mx[0], mx[1], mx[2]), mx[3]);
                         const float mnew = fmaxf(m, mtile * scale2); // finite: column 0 of a row is never masked
-                        float sum[8];
+                        const uint64_t nm2 = pack2(-mnew, -mnew);
+                        uint64_t sum2[4] = {pack2(l * ex2(m - mnew), 0.f), 0ull, 0ull, 0ull};
 #pragma unroll
-                        for (int c = 0; c < 8; ++c) sum[c] = 0.f;
-                        sum[0] = l * ex2(m - mnew);
-#pragma unroll
-                        for (int c = 0; c < QCOLS; ++c) sum[c & 7] += ex2(fmaf(v[c], scale2, -mnew));
-                        l = ((sum[0] + sum[1]) + (sum[2] + sum[3])) + ((sum[4] + sum[5]) + (sum[6] + sum[7]));
+                        for (int c = 0; c < QCOLS; c += 2) {
+                            float x0, x1;
+                            unpack2(ffma2(pack2(v[c], v[c + 1]), sc2, nm2), x0, x1);
+                            sum2[(c >> 1) & 3] = fadd2(sum2[(c >> 1) & 3], pack2(ex2(x0), ex2(x1)));
+                        }
+                        l = hsum2(fadd2(fadd2(sum2[0], sum2[1]), fadd2(sum2[2], sum2[3])));
                         m = mnew;
                     } else {
-                        const float* ls = sh.lse_s[cq][sub & 1];
+                        const uint64_t* nl = reinterpret_cast<const uint64_t*>(sh.nlse_s[warp][sub & 1]);
                         if (mask) {
 #pragma unroll
                             for (int c = 0; c < QCOLS; ++c)
@@ -397,11 +433,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         }
 #pragma unroll
                         for (int c = 0; c < QCOLS; c += 4) {
-                            const float4 l4 = *reinterpret_cast<const float4*>(ls + c);
-                            acc[c & 7] += ex2(fmaf(v[c], scale2, -l4.x));
-                            acc[(c + 1) & 7] += ex2(fmaf(v[c + 1], scale2, -l4.y));
-                            acc[(c + 2) & 7] += ex2(fmaf(v[c + 2], scale2, -l4.z));
-                            acc[(c + 3) & 7] += ex2(fmaf(v[c + 3], scale2, -l4.w));
+                            const ulonglong2 n4 = *reinterpret_cast<const ulonglong2*>(nl + (c >> 1));
+                            float x0, x1, x2, x3;
+                            unpack2(ffma2(pack2(v[c], v[c + 1]), sc2, n4.x), x0, x1);
+                            unpack2(ffma2(pack2(v[c + 2], v[c + 3]), sc2, n4.y), x2, x3);
+                            acc2[(c >> 1) & 3] = fadd2(acc2[(c >> 1) & 3], pack2(ex2(x0), ex2(x1)));
+                            acc2[((c >> 1) + 1) & 3] = fadd2(acc2[((c >> 1) + 1) & 3], pack2(ex2(x2), ex2(x3)));
                         }
                     }
                 }
@@ -409,7 +446,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             // ---- item end: combine the four column quarters (fixed order) and store
             const bool bad = (*abort_flag != 0);
             const int slot = n & 1;
-            const float mine = (pass == 1) ? l : ((acc[0] + acc[1]) + (acc[2] + acc[3])) + ((acc[4] + acc[5]) + (acc[6] + acc[7]));
+            const float mine = (pass == 1) ? l : hsum2(fadd2(fadd2(acc2[0], acc2[1]), fadd2(acc2[2], acc2[3])));
             if (cq > 0) { sh.part_m[slot][cq - 1][row] = m; sh.part_l[slot][cq - 1][row] = mine; }
             named_bar(5, NEPI_WARPS * 32);
             if (cq == 0) {
