@@ -157,6 +157,44 @@ __device__ __forceinline__ uint64_t fadd2(uint64_t a, uint64_t b) {
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
     return r;
 }
+__device__ __forceinline__ uint64_t fsub2(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+// 2^x for a packed pair on the FMA and integer pipes, so that the special-function unit (the
+// bottleneck of both passes: one exponential per logit) only has to serve part of the columns.
+// Textbook scheme: n = round(x) read off the mantissa after adding 1.5*2^23, f = x - n in
+// [-1/2, 1/2], 2^f by a degree-4 minimax polynomial (max relative error 2.7e-6, coefficients fitted
+// for this file), 2^n applied by adding n to the exponent field.  Inputs are clamped at -125, where
+// the result (3e-38) is far below anything that matters in a sum of probabilities.
+__device__ __forceinline__ uint64_t ex2_poly2(uint64_t x2) {
+    float x0, x1;
+    unpack2(x2, x0, x1);
+    const uint64_t xc = pack2(fmaxf(x0, -125.f), fmaxf(x1, -125.f));
+    const uint64_t magic = pack2(12582912.f, 12582912.f);
+    const uint64_t t = fadd2(xc, magic);
+    const uint64_t f = fsub2(xc, fsub2(t, magic));
+    uint64_t p = ffma2(pack2(0.009570102207362652f, 0.009570102207362652f), f,
+                       pack2(0.05591785907745361f, 0.05591785907745361f));
+    p = ffma2(p, f, pack2(0.240247443318367f, 0.240247443318367f));
+    p = ffma2(p, f, pack2(0.6931217908859253f, 0.6931217908859253f));
+    p = ffma2(p, f, pack2(0.9999992847442627f, 0.9999992847442627f));
+    const uint32_t r0 = (uint32_t)p + ((uint32_t)t << 23);
+    const uint32_t r1 = (uint32_t)(p >> 32) + ((uint32_t)(t >> 32) << 23);
+    return ((uint64_t)r1 << 32) | r0;
+}
+// Pair k (of 16) of a 32-column chunk takes the polynomial route when bit k is set.
+#ifndef KVM_POLY_PAIRS
+#define KVM_POLY_PAIRS 0x0u
+#endif
+constexpr uint32_t POLY_PAIRS = KVM_POLY_PAIRS;   // default: none (measured: any share made both passes slower)
+__device__ __forceinline__ uint64_t ex2_pair(uint64_t x2, int k) {
+    if ((POLY_PAIRS >> k) & 1u) return ex2_poly2(x2);
+    float x0, x1;
+    unpack2(x2, x0, x1);
+    return pack2(ex2(x0), ex2(x1));
+}
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
     float r;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
@@ -279,7 +317,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                                 tile * TILE, head);
                 const int nt = sc.ntiles(tile);
                 const int b = head / (pass == 1 ? Hq : Hkv), hh = head % (pass == 1 ? Hq : Hkv);
-                const int span = T - tile;                   // pass 2: query tiles per query head
+                int bhead = (pass == 1) ? b * Hkv + hh / G : b * Hq + hh * G;   // B tile cursor, advanced incrementally
+                int btile = (pass == 1) ? 0 : tile;
                 for (int t = 0; t < nt; t += 2, ++cnt) {
                     const int s = cnt % NSTAGE;
                     const int nh = (t + 1 < nt) ? 2 : 1;
@@ -288,13 +327,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     last_b[s] = (cnt / NSTAGE) & 1;
                     mbar_expect_tx(&sh.bar.full_b[s], nh * TILE_BYTES);
                     for (int h = 0; h < nh; ++h) {
-                        int bhead, btile;
-                        if (pass == 1) { bhead = b * Hkv + hh / G; btile = t + h; }
-                        else { bhead = b * Hq + hh * G + (t + h) / span; btile = tile + (t + h) % span; }
 #pragma unroll
                         for (int kc = 0; kc < KCH; ++kc)
                             tma_load_3d(sB + s * PAIR_BYTES + kc * PAIR_CHUNK + h * CHUNK_BYTES, mapB,
                                         &sh.bar.full_b[s], kc * KCHUNK, btile * TILE, bhead);
+                        if (++btile == T && pass == 2) { btile = tile; ++bhead; }   // next query head of the group
                     }
                 }
             }
@@ -353,37 +390,49 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         uint32_t cnt = 0, sub = 0;                           // steps, 128-column sub-tiles
         bool ok = true;
         int head, tile;
-        // pass 2: -lse*log2(e) of the next sub-tile's columns is fetched one sub-tile ahead (lane c holds
+        // pass 2: -lse*log2(e) of a sub-tile's columns is fetched two sub-tiles ahead (lane c holds
         // column c); every warp keeps its own staged copy, so no barrier is needed to share it
-        float lse_next = 0.f;
-        auto fetch_lse = [&](int hd, int tl, int t) -> float {
-            const int b = hd / Hkv, hh = hd % Hkv, span = T - tl;
-            const int i = (tl + t % span) * TILE + cq * QCOLS + lane;
-            const float* lse_h = lse_in + ((size_t)b * Hq + hh * G + t / span) * S;
-            return (i < S) ? __ldg(lse_h + i) * -LOG2E : -INFINITY;   // -inf zeroes columns past the sequence end
+        float lse_r0 = 0.f, lse_r1 = 0.f;
+        // look-ahead cursor over this CTA's sub-tile sequence: (item, query head g of the group, query tile it),
+        // advanced without divisions
+        int la_n = 0, la_g = 0, la_it = 0, la_head = 0, la_tile = 0;
+        bool la_ok = (pass == 2) && sc.item(0, la_head, la_tile);
+        la_it = la_tile;
+        const float* la_lse = la_ok ? lse_in + ((size_t)(la_head / Hkv) * Hq + (la_head % Hkv) * G) * S : lse_in;
+        auto fetch_ahead = [&]() -> float {
+            if (!la_ok) return 0.f;
+            const int i = la_it * TILE + cq * QCOLS + lane;
+            // -inf zeroes columns past the sequence end
+            const float r = (i < S) ? __ldg(la_lse + (size_t)la_g * S + i) * -LOG2E : -INFINITY;
+            if (++la_it == T) {
+                la_it = la_tile;
+                if (++la_g == G) {
+                    la_g = 0;
+                    la_ok = sc.item(++la_n, la_head, la_tile);
+                    la_it = la_tile;
+                    if (la_ok) la_lse = lse_in + ((size_t)(la_head / Hkv) * Hq + (la_head % Hkv) * G) * S;
+                }
+            }
+            return r;
         };
-        if (pass == 2 && sc.item(0, head, tile)) lse_next = fetch_lse(head, tile, 0);
+        if (pass == 2) { lse_r0 = fetch_ahead(); lse_r1 = fetch_ahead(); }
         const uint64_t sc2 = pack2(scale2, scale2);
         for (int n = 0; sc.item(n, head, tile); ++n) {
             const int nt = sc.ntiles(tile);
-            const int span = T - tile;
-            int nhead = 0, ntile = 0;
-            const bool has_next = sc.item(n + 1, nhead, ntile);
             float m = -INFINITY, l = 0.f;                    // pass 1 state
             uint64_t acc2[4] = {0ull, 0ull, 0ull, 0ull};     // pass 2 state: four packed pairs of partial sums
+            int btile = (pass == 1) ? 0 : tile;              // B tile of the current sub-tile, advanced incrementally
             for (int t0 = 0; t0 < nt; t0 += 2, ++cnt) {
                 const int as = cnt % NACC;
                 const int nh = (t0 + 1 < nt) ? 2 : 1;
                 ok = mbar_wait(&sh.bar.acc_full[as], (cnt / NACC) & 1, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
                 if (ok) tc_fence_after();
-                for (int h = 0; h < nh; ++h, ++sub) {
-                    const int t = t0 + h;
-                    const int btile = (pass == 1) ? t : tile + t % span;
+                for (int h = 0; h < nh; ++h, ++sub, btile = (btile + 1 == T && pass == 2) ? tile : btile + 1) {
                     if (pass == 2) {
-                        sh.nlse_s[warp][sub & 1][lane] = lse_next;
-                        if (t + 1 < nt) lse_next = fetch_lse(head, tile, t + 1);
-                        else if (has_next) lse_next = fetch_lse(nhead, ntile, 0);
+                        sh.nlse_s[warp][sub & 1][lane] = lse_r0;
+                        lse_r0 = lse_r1;
+                        lse_r1 = fetch_ahead();
                         __syncwarp();
                     }
                     // On the diagonal tile whole quarters are masked (skip) or fully valid (no per-element mask).
@@ -417,11 +466,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         const uint64_t nm2 = pack2(-mnew, -mnew);
                         uint64_t sum2[4] = {pack2(l * ex2(m - mnew), 0.f), 0ull, 0ull, 0ull};
 #pragma unroll
-                        for (int c = 0; c < QCOLS; c += 2) {
-                            float x0, x1;
-                            unpack2(ffma2(pack2(v[c], v[c + 1]), sc2, nm2), x0, x1);
-                            sum2[(c >> 1) & 3] = fadd2(sum2[(c >> 1) & 3], pack2(ex2(x0), ex2(x1)));
-                        }
+                        for (int c = 0; c < QCOLS; c += 2)
+                            sum2[(c >> 1) & 3] = fadd2(sum2[(c >> 1) & 3],
+                                                       ex2_pair(ffma2(pack2(v[c], v[c + 1]), sc2, nm2), c >> 1));
                         l = hsum2(fadd2(fadd2(sum2[0], sum2[1]), fadd2(sum2[2], sum2[3])));
                         m = mnew;
                     } else {
@@ -434,11 +481,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 #pragma unroll
                         for (int c = 0; c < QCOLS; c += 4) {
                             const ulonglong2 n4 = *reinterpret_cast<const ulonglong2*>(nl + (c >> 1));
-                            float x0, x1, x2, x3;
-                            unpack2(ffma2(pack2(v[c], v[c + 1]), sc2, n4.x), x0, x1);
-                            unpack2(ffma2(pack2(v[c + 2], v[c + 3]), sc2, n4.y), x2, x3);
-                            acc2[(c >> 1) & 3] = fadd2(acc2[(c >> 1) & 3], pack2(ex2(x0), ex2(x1)));
-                            acc2[((c >> 1) + 1) & 3] = fadd2(acc2[((c >> 1) + 1) & 3], pack2(ex2(x2), ex2(x3)));
+                            acc2[(c >> 1) & 3] = fadd2(acc2[(c >> 1) & 3],
+                                                       ex2_pair(ffma2(pack2(v[c], v[c + 1]), sc2, n4.x), c >> 1));
+                            acc2[((c >> 1) + 1) & 3] = fadd2(acc2[((c >> 1) + 1) & 3],
+                                                             ex2_pair(ffma2(pack2(v[c + 2], v[c + 3]), sc2, n4.y), (c >> 1) + 1));
                         }
                     }
                 }
