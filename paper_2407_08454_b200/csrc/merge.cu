@@ -9,8 +9,11 @@
 // their K and V rows into shared memory with two bulk copies, and
 //   phase 1  one lane group per token computes its weight g_j (the pivot row is
 //            taken from shared memory when it lies in the tile, else from L2);
-//   phase 2  one thread per (tensor, channel) walks the tile's tokens in order,
-//            adding g_j x_j, and flushes at every set boundary.
+//   phase 2  the tile is cut into short chunks of consecutive tokens; one lane
+//            group per (chunk, tensor) walks its chunk in order with 16-byte
+//            shared-memory reads, adding g_j x_j, and flushes at set boundaries;
+//   phase 3  sets that cross chunk boundaries are completed from per-chunk
+//            "head"/"tail" partial sums kept in shared memory.
 // A set that lies inside the tile is finished there.  A set that crosses tile
 // boundaries leaves fp32 partial sums in a scratch slot per (unit, tile): "head"
 // = the tile's tokens before its first boundary, "tail" = after its last; a small
@@ -61,29 +64,43 @@ template <int D> struct Slots {
     }
 };
 
+constexpr int MERGE_NT = 256;
+
+// Shared-memory footprint of the per-chunk partial sums (see merge_tile_kernel).
+template <typename T, int D> struct MergeGeom {
+    static constexpr int N = Vec<T>::N;              // elements per 16 bytes
+    static constexpr int LPR = D / N;                // lanes per row
+    static constexpr int NWORK = MERGE_NT / LPR;     // lane groups per block
+    static constexpr int NCH = NWORK / 2;            // token chunks per tile (one group per chunk and tensor)
+};
+
 template <typename T, int D, int TOK>
-__global__ void __launch_bounds__(2 * D) merge_tile_kernel(const T* __restrict__ K, const T* __restrict__ V,
-                                                           const int32_t* __restrict__ set_start,
-                                                           const int32_t* __restrict__ pivot,
-                                                           const int32_t* __restrict__ set_id,
-                                                           T* __restrict__ K_out, T* __restrict__ V_out,
-                                                           int32_t* __restrict__ out_size, Slots<D> slots, int S,
-                                                           int cap, float neg_inv_2s2_log2e, int scale_v) {
-    constexpr int N = Vec<T>::N;          // elements per 16 bytes
-    constexpr int LPR = D / N;            // lanes per row
-    constexpr int NT = 2 * D;             // threads: one per (tensor, channel)
-    constexpr int NWORK = NT / LPR;       // lane groups in phase 1
+__global__ void __launch_bounds__(MERGE_NT) merge_tile_kernel(const T* __restrict__ K, const T* __restrict__ V,
+                                                              const int32_t* __restrict__ set_start,
+                                                              const int32_t* __restrict__ pivot,
+                                                              const int32_t* __restrict__ set_id,
+                                                              T* __restrict__ K_out, T* __restrict__ V_out,
+                                                              int32_t* __restrict__ out_size, Slots<D> slots, int S,
+                                                              int cap, float neg_inv_2s2_log2e, int scale_v) {
+    using Gm = MergeGeom<T, D>;
+    constexpr int N = Gm::N, LPR = Gm::LPR, NWORK = Gm::NWORK, NCH = Gm::NCH;
+    constexpr int CHL = TOK / NCH;                    // tokens per chunk
+    static_assert(TOK % NCH == 0 && CHL >= 1, "tile must split evenly into chunks");
     extern __shared__ __align__(128) uint8_t smem_raw[];
     T* sK = reinterpret_cast<T*>(smem_raw);
     T* sV = sK + TOK * D;
+    // per-chunk partial sums: [chunk][head|tail][K|V][D]
+    float* sPart = reinterpret_cast<float*>(sV + TOK * D);
     __shared__ __align__(8) uint64_t bar;
     __shared__ int s_sid[TOK], s_piv[TOK], s_beg[TOK], s_end[TOK];
     __shared__ float s_g[TOK];
+    __shared__ float s_gpart[NCH][2];
 
     const int tile = blockIdx.x, Tn = gridDim.x;
     const long long u = blockIdx.y;
     const int tok0 = tile * TOK;
     const int ntok = min(TOK, S - tok0);
+    const int tile_end = tok0 + ntok;
     const T* Ku = K + (size_t)u * S * D;
     const T* Vu = V + (size_t)u * S * D;
     const int32_t* st = set_start + (size_t)u * (cap + 1);
@@ -100,7 +117,7 @@ __global__ void __launch_bounds__(2 * D) merge_tile_kernel(const T* __restrict__
                      ::"r"(smem_u32(sV)), "l"(Vu + (size_t)tok0 * D), "r"(bytes), "r"(smem_u32(&bar)) : "memory");
     }
     // per-token set data while the rows are in flight
-    for (int j = threadIdx.x; j < ntok; j += NT) {
+    for (int j = threadIdx.x; j < ntok; j += MERGE_NT) {
         const int sid = __ldg(set_id + (size_t)u * S + tok0 + j);
         s_sid[j] = sid;
         s_piv[j] = __ldg(pivot + (size_t)u * cap + sid);
@@ -116,62 +133,139 @@ __global__ void __launch_bounds__(2 * D) merge_tile_kernel(const T* __restrict__
                          "selp.u32 %0, 1, 0, p;\n\t}" : "=r"(done) : "r"(smem_u32(&bar)) : "memory");
     }
 
-    // ---- phase 1: weights
-    {
-        const int w = threadIdx.x / LPR, lane = threadIdx.x % LPR;
-        const unsigned gmask = (LPR == 32) ? 0xffffffffu : (((1u << LPR) - 1u) << ((threadIdx.x % 32) / LPR * LPR));
-        for (int j = w; j < ntok; j += NWORK) {
-            const int p = s_piv[j];
-            float kj[N], kp[N];
-            Vec<T>::unpack(*reinterpret_cast<const uint4*>(sK + (size_t)j * D + lane * N), kj);
-            if (p >= tok0 && p < tok0 + ntok)
-                Vec<T>::unpack(*reinterpret_cast<const uint4*>(sK + (size_t)(p - tok0) * D + lane * N), kp);
-            else
-                Vec<T>::unpack(ldg16(Ku + (size_t)p * D + lane * N), kp);
-            float d2 = 0.f;
+    const int w = threadIdx.x / LPR, lane = threadIdx.x % LPR;
+    const unsigned gmask = (LPR == 32) ? 0xffffffffu : (((1u << LPR) - 1u) << ((threadIdx.x % 32) / LPR * LPR));
+
+    // ---- phase 1: weights, one lane group per token
+    for (int j = w; j < ntok; j += NWORK) {
+        const int p = s_piv[j];
+        float kj[N], kp[N];
+        Vec<T>::unpack(*reinterpret_cast<const uint4*>(sK + (size_t)j * D + lane * N), kj);
+        if (p >= tok0 && p < tile_end)
+            Vec<T>::unpack(*reinterpret_cast<const uint4*>(sK + (size_t)(p - tok0) * D + lane * N), kp);
+        else
+            Vec<T>::unpack(ldg16(Ku + (size_t)p * D + lane * N), kp);
+        float d2 = 0.f;
 #pragma unroll
-            for (int e = 0; e < N; ++e) { const float a = kp[e] - kj[e]; d2 = fmaf(a, a, d2); }
+        for (int e = 0; e < N; ++e) { const float a = kp[e] - kj[e]; d2 = fmaf(a, a, d2); }
 #pragma unroll
-            for (int off = 1; off < LPR; off <<= 1) d2 += __shfl_xor_sync(gmask, d2, off);
-            if (lane == 0) s_g[j] = exp2f(d2 * neg_inv_2s2_log2e);
-        }
+        for (int off = 1; off < LPR; off <<= 1) d2 += __shfl_xor_sync(gmask, d2, off);
+        if (lane == 0) s_g[j] = exp2f(d2 * neg_inv_2s2_log2e);
     }
     __syncthreads();
 
-    // ---- phase 2: one thread per (tensor, channel) walks the tokens
-    const int which = threadIdx.x / D, ch = threadIdx.x % D;     // 0: K, 1: V
+    // ---- phase 2: lane group (chunk q, tensor) walks CHL consecutive tokens; a lane owns N channels
+    const int q = w >> 1, which = w & 1;                 // 0: K, 1: V
     const T* sX = which ? sV : sK;
     T* out = which ? V_out : K_out;
-    const int tile_end = tok0 + ntok;
-    float acc = 0.f, gs = 0.f;
-    T first_raw = sX[ch];
-    auto flush = [&](int j_last) {       // the set whose last token in this tile is j_last
-        const int sid = s_sid[j_last], beg = s_beg[j_last], end = s_end[j_last];
-        const bool started_here = beg >= tok0, closes_here = end <= tile_end;
-        if (started_here && closes_here) {
-            const int n = end - beg;
-            T r;
-            if (n == 1) r = first_raw;
-            else r = f32_to_elem<T>(which && scale_v ? acc * ((float)n / gs) : acc / gs);
-            out[((size_t)u * cap + sid) * D + ch] = r;
-            if (out_size && threadIdx.x == 0) out_size[(size_t)u * cap + sid] = n;
-        } else {
-            const int slot = started_here ? 1 : 0;               // tail : head
-            slots.s(u, Tn, tile, slot)[threadIdx.x] = acc;
-            if (threadIdx.x == 0) *slots.g(u, Tn, tile, slot) = gs;
+    float* partH = sPart + ((size_t)(q * 2 + 0) * 2 + which) * D + lane * N;
+    float* partL = sPart + ((size_t)(q * 2 + 1) * 2 + which) * D + lane * N;
+    const int c0 = q * CHL, c1 = min(c0 + CHL, ntok);     // chunk = tile tokens [c0, c1)
+    if (c0 < ntok) {
+        float acc[N], gs = 0.f;
+#pragma unroll
+        for (int e = 0; e < N; ++e) acc[e] = 0.f;
+        uint4 first_raw = *reinterpret_cast<const uint4*>(sX + (size_t)c0 * D + lane * N);
+        auto flush = [&](int j_last) {   // the set whose last token in this chunk is j_last (tile-relative)
+            const int sid = s_sid[j_last], beg = s_beg[j_last], end = s_end[j_last];
+            const bool started_here = beg >= tok0 + c0, closes_here = end <= tok0 + c1;
+            if (started_here && closes_here) {
+                const int n = end - beg;
+                uint4 r = first_raw;
+                if (n > 1) {
+                    const float mul = (which && scale_v) ? (float)n / gs : 1.f / gs;
+                    float o[N];
+#pragma unroll
+                    for (int e = 0; e < N; ++e) o[e] = acc[e] * mul;
+                    r = Vec<T>::pack(o);
+                }
+                *reinterpret_cast<uint4*>(out + ((size_t)u * cap + sid) * D + lane * N) = r;
+                if (out_size && which == 0 && lane == 0) out_size[(size_t)u * cap + sid] = n;
+            } else {
+                float* dst = started_here ? partL : partH;
+#pragma unroll
+                for (int e = 0; e < N; ++e) dst[e] = acc[e];
+                if (which == 0 && lane == 0) s_gpart[q][started_here ? 1 : 0] = gs;
+            }
+        };
+        for (int j = c0; j < c1; ++j) {
+            const uint4 raw = *reinterpret_cast<const uint4*>(sX + (size_t)j * D + lane * N);
+            if (j > c0 && s_sid[j] != s_sid[j - 1]) {
+                flush(j - 1);
+#pragma unroll
+                for (int e = 0; e < N; ++e) acc[e] = 0.f;
+                gs = 0.f;
+                first_raw = raw;
+            }
+            const float g = s_g[j];
+            float x[N];
+            Vec<T>::unpack(raw, x);
+#pragma unroll
+            for (int e = 0; e < N; ++e) acc[e] = fmaf(g, x[e], acc[e]);
+            gs += g;
         }
-    };
-    for (int j = 0; j < ntok; ++j) {
-        if (j > 0 && s_sid[j] != s_sid[j - 1]) {
-            flush(j - 1);
-            acc = 0.f; gs = 0.f;
-            first_raw = sX[(size_t)j * D + ch];
-        }
-        const float g = s_g[j];
-        acc = fmaf(g, elem_to_f32<T>(sX[(size_t)j * D + ch]), acc);
-        gs += g;
+        flush(c1 - 1);
     }
-    flush(ntok - 1);
+    __syncthreads();
+
+    // ---- phase 3: sets that cross chunk boundaries.  Boundary q (the start of chunk q; q = 0 is the
+    // tile start) is handled by the same lane group: if a set crosses it and does not cross the next
+    // one, its pieces (tail of the chunk where it began, heads of the chunks it covers) are added in
+    // chunk order and stored as the finished row, or as this tile's head / tail slot when the set
+    // extends beyond the tile.
+    if (c0 < ntok) {
+        const int beg = s_beg[c0], end = s_end[c0], sid = s_sid[c0];
+        const int tokb = tok0 + c0;
+        const bool crosses = beg < tokb;
+        const bool last_in_tile = (tok0 + c1 == tile_end);
+        if (crosses && (end <= tok0 + c1 || last_in_tile)) {
+            float sum[N], gs = 0.f;
+#pragma unroll
+            for (int e = 0; e < N; ++e) sum[e] = 0.f;
+            int qa = 0;
+            if (beg >= tok0) {                               // began in this tile: its chunk holds a tail piece
+                qa = (beg - tok0) / CHL;
+                const float* pl = sPart + ((size_t)(qa * 2 + 1) * 2 + which) * D + lane * N;
+#pragma unroll
+                for (int e = 0; e < N; ++e) sum[e] = pl[e];
+                gs = s_gpart[qa][1];
+                ++qa;
+            }
+            for (int c = qa; c <= q; ++c) {
+                const float* ph = sPart + ((size_t)(c * 2 + 0) * 2 + which) * D + lane * N;
+#pragma unroll
+                for (int e = 0; e < N; ++e) sum[e] += ph[e];
+                gs += s_gpart[c][0];
+            }
+            if (beg >= tok0 && end <= tile_end) {            // whole set inside the tile: finished row
+                const int n = end - beg;
+                const float mul = (which && scale_v) ? (float)n / gs : 1.f / gs;
+                float o[N];
+#pragma unroll
+                for (int e = 0; e < N; ++e) o[e] = sum[e] * mul;
+                *reinterpret_cast<uint4*>(out + ((size_t)u * cap + sid) * D + lane * N) = Vec<T>::pack(o);
+                if (out_size && which == 0 && lane == 0) out_size[(size_t)u * cap + sid] = n;
+            } else {
+                const int slot = (beg >= tok0) ? 1 : 0;      // tail : head of this tile
+                float* dst = slots.s(u, Tn, tile, slot) + which * D + lane * N;
+#pragma unroll
+                for (int e = 0; e < N; ++e) dst[e] = sum[e];
+                if (which == 0 && lane == 0) *slots.g(u, Tn, tile, slot) = gs;
+            }
+        }
+        // a set that begins inside the tile's last chunk and runs past the tile: its tail piece is the tile's tail
+        if (last_in_tile) {
+            const int jl = c1 - 1;
+            const int bl = s_beg[jl], el = s_end[jl];
+            if (bl >= tokb && el > tile_end) {
+                const float* pl = sPart + ((size_t)(q * 2 + 1) * 2 + which) * D + lane * N;
+                float* dst = slots.s(u, Tn, tile, 1) + which * D + lane * N;
+#pragma unroll
+                for (int e = 0; e < N; ++e) dst[e] = pl[e];
+                if (which == 0 && lane == 0) *slots.g(u, Tn, tile, 1) = s_gpart[q][1];
+            }
+        }
+    }
 }
 
 // Sets that cross a tile boundary: the block of the LAST boundary a set crosses adds its slots in tile order.
@@ -213,12 +307,12 @@ cudaError_t launch_t(const Dims& d, const void* K, const void* V, const int32_t*
     Slots<D> slots;
     slots.sums = scratch;
     slots.gsum = scratch + (size_t)d.U * Tn * 2 * (2 * D);
-    const size_t smem = (size_t)2 * TOK * D * sizeof(T);
+    const size_t smem = (size_t)2 * TOK * D * sizeof(T) + (size_t)MergeGeom<T, D>::NCH * 2 * 2 * D * sizeof(float);
     cudaError_t e = cudaFuncSetAttribute(merge_tile_kernel<T, D, TOK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)smem);
     if (e != cudaSuccess) return e;
     const float c = -LOG2E / (2.f * d.sigma * d.sigma);
-    merge_tile_kernel<T, D, TOK><<<dim3(Tn, d.U), 2 * D, smem, st>>>(
+    merge_tile_kernel<T, D, TOK><<<dim3(Tn, d.U), MERGE_NT, smem, st>>>(
         (const T*)K, (const T*)V, set_start, pivot, set_id, (T*)K_out, (T*)V_out, out_size, slots, d.S, d.cap, c,
         d.scale_v);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
