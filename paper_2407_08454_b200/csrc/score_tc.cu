@@ -402,8 +402,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         auto fetch_ahead = [&]() -> float {
             if (!la_ok) return 0.f;
             const int i = la_it * TILE + cq * QCOLS + lane;
-            // -inf zeroes columns past the sequence end
-            const float r = (i < S) ? __ldg(la_lse + (size_t)la_g * S + i) * -LOG2E : -INFINITY;
+            // the raw value is kept untouched until it is staged, so that nothing waits on the load here;
+            // +inf (staged as -inf) zeroes columns past the sequence end
+            const float r = (i < S) ? __ldg(la_lse + (size_t)la_g * S + i) : INFINITY;
             if (++la_it == T) {
                 la_it = la_tile;
                 if (++la_g == G) {
@@ -430,7 +431,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 if (ok) tc_fence_after();
                 for (int h = 0; h < nh; ++h, ++sub, btile = (btile + 1 == T && pass == 2) ? tile : btile + 1) {
                     if (pass == 2) {
-                        sh.nlse_s[warp][sub & 1][lane] = lse_r0;
+                        sh.nlse_s[warp][sub & 1][lane] = lse_r0 * -LOG2E;
                         lse_r0 = lse_r1;
                         lse_r1 = fetch_ahead();
                         __syncwarp();

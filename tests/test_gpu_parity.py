@@ -103,6 +103,38 @@ def test_c1_llama2_7b_layer_full():
     assert g.stats.status == 0
 
 
+def _full_config_check(name, layer, sample_units):
+    """One layer of a full-size workload: every unit through the library, invariants on every unit,
+    the fp64 checker on a seeded sample of units."""
+    cfg = si.CONFIGS[name]
+    case = _case(cfg, layer=layer)
+    g = run_gpu(case)
+    assert g.stats.status == 0
+    check_invariants_all_units(case, g)
+    rep = check_case(case, g, units=sample_units)
+    print(name, "layer", layer, rep, "budget-rule units", g.stats.units_budget_rule, "near-threshold pairs",
+          g.stats.near_threshold, "out_len", g.stats.min_out_len, g.stats.max_out_len)
+    return g, rep
+
+
+def test_c2_llama2_7b_full_cache_layer():
+    # batch 4 x 32 heads = 128 units, 35 % budget, per-layer rho (layer 5 draws a low one: many similarity cuts)
+    rng = np.random.default_rng(2)
+    _full_config_check("C2", 5, sorted(rng.choice(128, 8, replace=False).tolist()))
+
+
+def test_c3_mistral_gqa_32k_layer():
+    # 8 KV heads x 4 query heads, 32768 tokens; the checker runs one whole GQA group
+    g, rep = _full_config_check("C3", 0, [3])
+    assert g.cap == 16384
+
+
+def test_c4_llama2_13b_layer():
+    # batch 8 x 40 heads = 320 units, keys with regime switches (many short sets), 35 % budget
+    rng = np.random.default_rng(4)
+    _full_config_check("C4", 1, sorted(rng.choice(320, 8, replace=False).tolist()))
+
+
 def test_compress_is_reproducible_bit_for_bit():
     case = _case(si.CONFIGS["C1"].scaled(seq=1536, n_q_heads=4, n_kv_heads=4, seed=11))
     a, b = run_gpu(case), run_gpu(case)
