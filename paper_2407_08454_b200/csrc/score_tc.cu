@@ -15,8 +15,8 @@
 // attention map in registers, with no cross-lane reduction.
 //
 // One CTA per SM, persistent, warp-specialised:
-//   warps 0-15 epilogue: tcgen05.ld the accumulator (warp w reads TMEM lanes
-//              32*(w%4).., column quarter w/4), exp2 on the SFUs, row/column state
+//   warps 0-15 epilogue: two groups of 8 take alternate steps; a warp reads TMEM lanes
+//              32*(w%4).. and one column half, does exp2 on the SFUs, keeps row/column state
 //   warp  16   producer: TMA (cp.async.bulk.tensor, 128B swizzle) into a 2-stage ring of B pairs
 //   warp  17   MMA issue: one thread issues tcgen05.mma / tcgen05.commit; owns TMEM
 // Work items are dealt in descending length, boustrophedon over the CTAs, which
@@ -242,6 +242,31 @@ struct Sched {
     __device__ __forceinline__ int ntiles(int tile) const { return (pass == 1) ? tile + 1 : G * (T - tile); }
 };
 
+// Walks a CTA's steps (pairs of B tiles) across its items; (bg, bt) = query head within the group and
+// query tile of the step's first B tile in pass 2, advanced without divisions.
+struct StepIter {
+    int n, t0, head, tile, nt, bg, bt;
+    uint32_t cnt;
+    bool valid;
+    __device__ __forceinline__ void load(const Sched& sc) {
+        valid = sc.item(n, head, tile);
+        nt = valid ? sc.ntiles(tile) : 0;
+        t0 = 0; bg = 0; bt = tile;
+    }
+    __device__ __forceinline__ void init(const Sched& sc) { n = 0; cnt = 0; load(sc); }
+    __device__ __forceinline__ void next(const Sched& sc) {
+        if (!valid) return;
+        ++cnt;
+        t0 += 2;
+        if (t0 >= nt) { ++n; load(sc); return; }
+        if (sc.pass == 2) {
+#pragma unroll
+            for (int i = 0; i < 2; ++i)
+                if (++bt == sc.T) { bt = tile; ++bg; }
+        }
+    }
+};
+
 struct __align__(8) Barriers {
     uint64_t full_a[2], empty_a[2];
     uint64_t full_b[NSTAGE], empty_b[NSTAGE];
@@ -252,10 +277,10 @@ struct alignas(16) Shared {
     Barriers bar;
     uint32_t tmem_base;
     int abort_flag;
-    float part_m[2][3][TILE];    // partials of column quarters 1..3 at item end, double-buffered by item parity
+    float part_m[2][3][TILE];    // row states of warp sets 1..3 at item end, double-buffered by item parity
     float part_l[2][3][TILE];
-    alignas(16) float nlse_s[NEPI_WARPS][2][QCOLS];   // pass 2: each warp's own copy of -lse*log2(e) of its 32
-                                                      // columns, double-buffered by sub-tile parity
+    alignas(16) float nlse_s[NEPI_WARPS][2][128];     // pass 2: each warp's own copy of -lse*log2(e) of its 64
+                                                      // columns of both sub-tiles of a step, double-buffered
 };
 
 template <int KCH>
@@ -283,7 +308,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     if (threadIdx.x == 0) {
         for (int i = 0; i < 2; ++i) { mbar_init(&sh.bar.full_a[i], 1); mbar_init(&sh.bar.empty_a[i], 1); }
         for (int i = 0; i < NSTAGE; ++i) { mbar_init(&sh.bar.full_b[i], 1); mbar_init(&sh.bar.empty_b[i], 1); }
-        for (int i = 0; i < NACC; ++i) { mbar_init(&sh.bar.acc_full[i], 1); mbar_init(&sh.bar.acc_empty[i], NEPI_WARPS); }
+        for (int i = 0; i < NACC; ++i) { mbar_init(&sh.bar.acc_full[i], 1); mbar_init(&sh.bar.acc_empty[i], NEPI_WARPS / 2); }
         sh.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -383,127 +408,153 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         }
     } else {
         // ============================== epilogue ==============================
+        // Two groups of 8 warps take alternate steps (group g always reads accumulator stage g), so that
+        // one group's waits, TMEM loads and bookkeeping overlap the other group's exponentials.  Within a
+        // group a warp owns TMEM lane quarter lq and one 64-column half of each 128-column sub-tile,
+        // handled as two 32-column chunks.
         const int lq = warp & 3;                             // TMEM lane quarter this warp may read
-        const int cq = warp >> 2;                            // column quarter of every 128-column sub-tile
+        const int grp = (warp >> 2) & 1;                     // steps with (cnt & 1) == grp
+        const int chalf = warp >> 3;                         // column half of a sub-tile
+        const int pidx = warp >> 2;                          // partial-sum slot of this warp's row state (0..3)
         const int row = lq * 32 + lane;                      // A row = TMEM lane
-        const uint32_t t_lane = tmem_base + ((uint32_t)(lq * 32) << 16) + cq * QCOLS;
-        uint32_t cnt = 0, sub = 0;                           // steps, 128-column sub-tiles
-        bool ok = true;
-        int head, tile;
-        // pass 2: -lse*log2(e) of a sub-tile's columns is fetched two sub-tiles ahead (lane c holds
-        // column c); every warp keeps its own staged copy, so no barrier is needed to share it
-        float lse_r0 = 0.f, lse_r1 = 0.f;
-        // look-ahead cursor over this CTA's sub-tile sequence: (item, query head g of the group, query tile it),
-        // advanced without divisions
-        int la_n = 0, la_g = 0, la_it = 0, la_head = 0, la_tile = 0;
-        bool la_ok = (pass == 2) && sc.item(0, la_head, la_tile);
-        la_it = la_tile;
-        const float* la_lse = la_ok ? lse_in + ((size_t)(la_head / Hkv) * Hq + (la_head % Hkv) * G) * S : lse_in;
-        auto fetch_ahead = [&]() -> float {
-            if (!la_ok) return 0.f;
-            const int i = la_it * TILE + cq * QCOLS + lane;
-            // the raw value is kept untouched until it is staged, so that nothing waits on the load here;
-            // +inf (staged as -inf) zeroes columns past the sequence end
-            const float r = (i < S) ? __ldg(la_lse + (size_t)la_g * S + i) : INFINITY;
-            if (++la_it == T) {
-                la_it = la_tile;
-                if (++la_g == G) {
-                    la_g = 0;
-                    la_ok = sc.item(++la_n, la_head, la_tile);
-                    la_it = la_tile;
-                    if (la_ok) la_lse = lse_in + ((size_t)(la_head / Hkv) * Hq + (la_head % Hkv) * G) * S;
-                }
-            }
-            return r;
-        };
-        if (pass == 2) { lse_r0 = fetch_ahead(); lse_r1 = fetch_ahead(); }
+        const uint32_t t_lane = tmem_base + ((uint32_t)(lq * 32) << 16) + grp * ACC_COLS + chalf * 64;
         const uint64_t sc2 = pack2(scale2, scale2);
-        for (int n = 0; sc.item(n, head, tile); ++n) {
-            const int nt = sc.ntiles(tile);
+        bool ok = true;
+        StepIter it;
+        it.init(sc);
+        // pass 2: the row-lse values of this warp's 64 columns are fetched one own-step ahead (lane c holds
+        // columns c and c + 32 of its half, for both sub-tiles of the step) and staged per warp
+        float lse_nx[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+        auto fetch_step = [&](const StepIter& w) {
+            int g = w.bg, q = w.bt;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const float* lse_h = lse_in + ((size_t)(w.head / Hkv) * Hq + (w.head % Hkv) * G + g) * S;
+                const int i0 = q * TILE + chalf * 64 + lane;
+                const bool live = w.valid && (w.t0 + h < w.nt);
+                // raw values; +inf (staged as -inf) zeroes columns past the sequence end
+                lse_nx[h][0] = (live && i0 < S) ? __ldg(lse_h + i0) : INFINITY;
+                lse_nx[h][1] = (live && i0 + 32 < S) ? __ldg(lse_h + i0 + 32) : INFINITY;
+                if (++q == T) { q = w.tile; ++g; }
+            }
+        };
+        if (pass == 2) {
+            StepIter la = it;
+            if (grp == 1) la.next(sc);
+            fetch_step(la);
+        }
+        uint32_t own = 0;                                    // own steps processed (accumulator phase, staging parity)
+        while (it.valid) {
+            const int n = it.n, head = it.head, tile = it.tile;
             float m = -INFINITY, l = 0.f;                    // pass 1 state
-            uint64_t acc2[4] = {0ull, 0ull, 0ull, 0ull};     // pass 2 state: four packed pairs of partial sums
-            int btile = (pass == 1) ? 0 : tile;              // B tile of the current sub-tile, advanced incrementally
-            for (int t0 = 0; t0 < nt; t0 += 2, ++cnt) {
-                const int as = cnt % NACC;
-                const int nh = (t0 + 1 < nt) ? 2 : 1;
-                ok = mbar_wait(&sh.bar.acc_full[as], (cnt / NACC) & 1, abort_flag);
+            float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};   // pass 2 state: eight partial sums
+            for (; it.valid && it.n == n; it.next(sc)) {
+                if ((int)(it.cnt & 1u) != grp) continue;
+                const int nh = (it.t0 + 1 < it.nt) ? 2 : 1;
+                if (pass == 2) {
+                    // stage this step's values (scaled to -lse*log2 e), then start the loads for the next own step
+                    float* stg = sh.nlse_s[warp][own & 1];
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        stg[h * 64 + lane] = lse_nx[h][0] * -LOG2E;
+                        stg[h * 64 + 32 + lane] = lse_nx[h][1] * -LOG2E;
+                    }
+                    StepIter la = it;
+                    la.next(sc);
+                    la.next(sc);
+                    fetch_step(la);
+                    __syncwarp();
+                }
+                ok = mbar_wait(&sh.bar.acc_full[grp], own & 1, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
                 if (ok) tc_fence_after();
-                for (int h = 0; h < nh; ++h, ++sub, btile = (btile + 1 == T && pass == 2) ? tile : btile + 1) {
-                    if (pass == 2) {
-                        sh.nlse_s[warp][sub & 1][lane] = lse_r0 * -LOG2E;
-                        lse_r0 = lse_r1;
-                        lse_r1 = fetch_ahead();
-                        __syncwarp();
-                    }
-                    // On the diagonal tile whole quarters are masked (skip) or fully valid (no per-element mask).
+                int btile = (pass == 1) ? it.t0 : it.bt;
+                for (int h = 0; h < nh; ++h) {
                     const bool diag = (btile == tile);
-                    const bool skip = diag && ((pass == 1) ? (cq > lq) : (cq < lq));
-                    const bool mask = diag && (cq == lq);
-                    float v[QCOLS];
-                    if (ok && !skip) tmem_ld32(t_lane + as * ACC_COLS + h * TILE, v);
-                    if (h == nh - 1) {                       // last read of this accumulator: release it
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(&sh.bar.acc_empty[as]);
+#pragma unroll
+                    for (int k = 0; k < 2; ++k) {
+                        const int cq = chalf * 2 + k;            // column quarter of this 32-column chunk
+                        // On the diagonal tile whole quarters are masked (skip) or fully valid (no per-element mask).
+                        const bool skip = diag && ((pass == 1) ? (cq > lq) : (cq < lq));
+                        const bool mask = diag && (cq == lq);
+                        float v[QCOLS];
+                        if (ok && !skip) tmem_ld32(t_lane + h * TILE + k * QCOLS, v);
+                        if (h == nh - 1 && k == 1) {         // last read of this accumulator: release it
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(&sh.bar.acc_empty[grp]);
+                        }
+                        if (!ok || skip) continue;
+                        if (pass == 1) {
+                            if (mask) {
+#pragma unroll
+                                for (int c = 0; c < QCOLS; ++c)
+                                    if (c > lane) v[c] = -INFINITY;      // key after query
+                            }
+                            float mx[4];
+#pragma unroll
+                            for (int c = 0; c < 4; ++c) {
+                                mx[c] = fmax3(v[c], v[c + 4], v[c + 8]);
+                                mx[c] = fmax3(mx[c], v[c + 12], v[c + 16]);
+                                mx[c] = fmax3(mx[c], v[c + 20], v[c + 24]);
+                                mx[c] = fmaxf(mx[c], v[c + 28]);
+                            }
+                            const float mtile = fmaxf(fmax3(mx[0], mx[1], mx[2]), mx[3]);
+                            const float mnew = fmaxf(m, mtile * scale2);
+                            if (mnew > -INFINITY) {
+                                const uint64_t nm2 = pack2(-mnew, -mnew);
+                                // packed multiply-add for the exponents (the accumulator registers come in
+                                // adjacent pairs); the exponentials are summed in eight scalar chains
+                                float sum[8] = {l * ex2(m - mnew), 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                                for (int c = 0; c < QCOLS; c += 2) {
+                                    float e0, e1;
+                                    unpack2(ex2_pair(ffma2(pack2(v[c], v[c + 1]), sc2, nm2), c >> 1), e0, e1);
+                                    sum[c & 7] += e0;
+                                    sum[(c + 1) & 7] += e1;
+                                }
+                                l = ((sum[0] + sum[1]) + (sum[2] + sum[3])) + ((sum[4] + sum[5]) + (sum[6] + sum[7]));
+                                m = mnew;
+                            }
+                        } else {
+                            const uint64_t* nl =
+                                reinterpret_cast<const uint64_t*>(sh.nlse_s[warp][own & 1] + h * 64 + k * QCOLS);
+                            if (mask) {
+#pragma unroll
+                                for (int c = 0; c < QCOLS; ++c)
+                                    if (c < lane) v[c] = -INFINITY;      // query before key
+                            }
+#pragma unroll
+                            for (int c = 0; c < QCOLS; c += 4) {
+                                const ulonglong2 n4 = *reinterpret_cast<const ulonglong2*>(nl + (c >> 1));
+                                float e0, e1, e2, e3;
+                                unpack2(ex2_pair(ffma2(pack2(v[c], v[c + 1]), sc2, n4.x), c >> 1), e0, e1);
+                                unpack2(ex2_pair(ffma2(pack2(v[c + 2], v[c + 3]), sc2, n4.y), (c >> 1) + 1), e2, e3);
+                                acc[c & 7] += e0;
+                                acc[(c + 1) & 7] += e1;
+                                acc[(c + 2) & 7] += e2;
+                                acc[(c + 3) & 7] += e3;
+                            }
+                        }
                     }
-                    if (!ok || skip) continue;
-                    if (pass == 1) {
-                        if (mask) {
-#pragma unroll
-                            for (int c = 0; c < QCOLS; ++c)
-                                if (c > lane) v[c] = -INFINITY;      // key after query
-                        }
-                        float mx[4];
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            mx[c] = fmax3(v[c], v[c + 4], v[c + 8]);
-                            mx[c] = fmax3(mx[c], v[c + 12], v[c + 16]);
-                            mx[c] = fmax3(mx[c], v[c + 20], v[c + 24]);
-                            mx[c] = fmaxf(mx[c], v[c + 28]);
-                        }
-                        const float mtile = fmaxf(fmax3(mx[0], mx[1], mx[2]), mx[3]);
-                        const float mnew = fmaxf(m, mtile * scale2); // finite: column 0 of a row is never masked
-                        const uint64_t nm2 = pack2(-mnew, -mnew);
-                        uint64_t sum2[4] = {pack2(l * ex2(m - mnew), 0.f), 0ull, 0ull, 0ull};
-#pragma unroll
-                        for (int c = 0; c < QCOLS; c += 2)
-                            sum2[(c >> 1) & 3] = fadd2(sum2[(c >> 1) & 3],
-                                                       ex2_pair(ffma2(pack2(v[c], v[c + 1]), sc2, nm2), c >> 1));
-                        l = hsum2(fadd2(fadd2(sum2[0], sum2[1]), fadd2(sum2[2], sum2[3])));
-                        m = mnew;
-                    } else {
-                        const uint64_t* nl = reinterpret_cast<const uint64_t*>(sh.nlse_s[warp][sub & 1]);
-                        if (mask) {
-#pragma unroll
-                            for (int c = 0; c < QCOLS; ++c)
-                                if (c < lane) v[c] = -INFINITY;      // query before key
-                        }
-#pragma unroll
-                        for (int c = 0; c < QCOLS; c += 4) {
-                            const ulonglong2 n4 = *reinterpret_cast<const ulonglong2*>(nl + (c >> 1));
-                            acc2[(c >> 1) & 3] = fadd2(acc2[(c >> 1) & 3],
-                                                       ex2_pair(ffma2(pack2(v[c], v[c + 1]), sc2, n4.x), c >> 1));
-                            acc2[((c >> 1) + 1) & 3] = fadd2(acc2[((c >> 1) + 1) & 3],
-                                                             ex2_pair(ffma2(pack2(v[c + 2], v[c + 3]), sc2, n4.y), (c >> 1) + 1));
-                        }
-                    }
+                    if (++btile == T && pass == 2) btile = tile;
                 }
+                ++own;
             }
-            // ---- item end: combine the four column quarters (fixed order) and store
+            // ---- item end: combine the four partial states of every row (fixed order) and store
             const bool bad = (*abort_flag != 0);
             const int slot = n & 1;
-            const float mine = (pass == 1) ? l : hsum2(fadd2(fadd2(acc2[0], acc2[1]), fadd2(acc2[2], acc2[3])));
-            if (cq > 0) { sh.part_m[slot][cq - 1][row] = m; sh.part_l[slot][cq - 1][row] = mine; }
+            const float mine = (pass == 1) ? l : ((acc[0] + acc[1]) + (acc[2] + acc[3])) + ((acc[4] + acc[5]) + (acc[6] + acc[7]));
+            if (pidx > 0) { sh.part_m[slot][pidx - 1][row] = m; sh.part_l[slot][pidx - 1][row] = mine; }
             named_bar(5, NEPI_WARPS * 32);
-            if (cq == 0) {
+            if (pidx == 0) {
                 const int gi = tile * TILE + row;
                 if (gi < S) {
                     if (pass == 1) {
                         float M = m;
 #pragma unroll
                         for (int q = 0; q < 3; ++q) M = fmaxf(M, sh.part_m[slot][q][row]);
-                        float L = l * ex2(m - M);                    // quarter 0 always holds column 0: m finite
+                        float L = (m > -INFINITY) ? l * ex2(m - M) : 0.f;
 #pragma unroll
                         for (int q = 0; q < 3; ++q) {
                             const float mq = sh.part_m[slot][q][row], lq_ = sh.part_l[slot][q][row];
