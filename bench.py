@@ -34,6 +34,9 @@ WORKLOAD = "C1"
 METRIC = "KV tokens compressed/s (all layers, heads)"
 UNIT = "KV tokens/s"
 N_BUFFERS = 3  # rotating input sets: 3 x 100 MB > 126 MB of L2
+# dram__bytes_read.sum + dram__bytes_write.sum of one column-pass launch on this workload, from the ncu capture
+# summarised in profiles/score_tc_column_pass_C1.md (set to None when the kernel changes until it is re-captured)
+NCU_TRAFFIC_BYTES_COLUMN_PASS = 67.74e6 + 2.30e6
 
 
 def measured_peaks():
@@ -265,7 +268,7 @@ def main():
     merge_bytes = 2 * work["k_bytes"] + 2 * out_rows * cfg.head_dim * 2
     roofline = {
         "kernel": "score column pass (kvm_score with lse_in)", "bound": "tensor", "achieved": achieved,
-        "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"], "traffic": None,
+        "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"], "traffic": NCU_TRAFFIC_BYTES_COLUMN_PASS,
         "peak_source": peaks["source"] + " burst bf16",
     }
     kernels = {
