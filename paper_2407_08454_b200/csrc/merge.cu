@@ -326,9 +326,14 @@ cudaError_t launch_t(const Dims& d, const void* K, const void* V, const int32_t*
 
 }  // namespace
 
-// Tokens per tile: 128 for 2-byte elements, 64 for 4-byte ones (64 KB resp. 32-64 KB of shared memory).
+// Tokens per tile.
+#ifndef KVM_MERGE_TOK_BF16
+#define KVM_MERGE_TOK_BF16 64
+#endif
+static int merge_tile_tokens(const Dims& d) { return d.dtype == KVM_BF16 ? KVM_MERGE_TOK_BF16 : 64; }
+
 size_t merge_scratch_floats(const Dims& d) {
-    const int TOK = d.dtype == KVM_BF16 ? 128 : 64;
+    const int TOK = merge_tile_tokens(d);
     const size_t Tn = (d.S + TOK - 1) / TOK;
     return (size_t)d.U * Tn * 2 * (2 * d.D) + (size_t)d.U * Tn * 2;
 }
@@ -343,9 +348,9 @@ cudaError_t launch_merge(const Dims& d, const void* K, const void* V, const int3
                          const int32_t* pivot, const int32_t* set_id, void* K_out, void* V_out, int32_t* out_size,
                          float* scratch, cudaStream_t st) {
     if (d.dtype == KVM_BF16) {
-        return d.D == 128 ? launch_t<__nv_bfloat16, 128, 128>(d, K, V, set_start, pivot, set_id, K_out, V_out,
+        return d.D == 128 ? launch_t<__nv_bfloat16, 128, KVM_MERGE_TOK_BF16>(d, K, V, set_start, pivot, set_id, K_out, V_out,
                                                               out_size, scratch, st)
-                          : launch_t<__nv_bfloat16, 64, 128>(d, K, V, set_start, pivot, set_id, K_out, V_out,
+                          : launch_t<__nv_bfloat16, 64, KVM_MERGE_TOK_BF16>(d, K, V, set_start, pivot, set_id, K_out, V_out,
                                                              out_size, scratch, st);
     }
     return d.D == 128
