@@ -57,7 +57,7 @@ enum kvm_status {
     KVM_E_UNSUPPORTED = -7, /* valid request this build cannot run (e.g. non-causal) */
     KVM_E_CUDA = -8,        /* the CUDA runtime refused a launch, a copy or a driver lookup */
     KVM_E_DEVICE_TIMEOUT = -9, /* only ever appears in kvm_stats.status: a bounded device wait gave up */
-    KVM_E_STATIC_LIMIT = -10 /* kvm_score_static: batch * n_q_heads * seq exceeds KVM_STATIC_SCORE_ROWS */
+    KVM_E_STATIC_LIMIT = -10 /* kvm_score_static: the problem does not fit the built-in scratch (see KVM_STATIC_SCORE_ROWS) */
 };
 
 /* The paper's problem statement as a plain struct (Section 2.4; hyper-parameters of Section 5.1). */
@@ -182,7 +182,8 @@ int kvm_compress_host(const kvm_params* p, const void* Q, const void* K, const v
  * until the process exits, whether or not this function is ever called.
  *
  *   - Same Q, K, scores and stream arguments as kvm_score; no lse_in, no ws.
- *   - batch * n_q_heads * seq must not exceed KVM_STATIC_SCORE_ROWS, otherwise
+ *   - batch * n_q_heads * seq must not exceed KVM_STATIC_SCORE_ROWS for fp32 tensors and
+ *     KVM_STATIC_SCORE_ROWS / 8 for bf16 tensors (their row pass leaves 32 bytes per row), otherwise
  *     KVM_E_STATIC_LIMIT is returned and nothing is enqueued.
  *   - The first call on each device looks up the array's device address (a
  *     one-time host-side set-up, done with that device current).  Make that first

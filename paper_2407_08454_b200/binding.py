@@ -133,7 +133,8 @@ def kvm_score(p: KvmParams, Q, K, lse_in, scores, ws, stream=None) -> None:
 
 def kvm_score_static(p: KvmParams, Q, K, scores, stream=None) -> None:
     """kvm_score on the library's built-in scratch: for callers that cannot allocate a workspace.
-    batch * n_q_heads * seq must not exceed KVM_STATIC_SCORE_ROWS; calls on one device must not overlap."""
+    batch * n_q_heads * seq must not exceed KVM_STATIC_SCORE_ROWS (fp32) or an eighth of it (bf16); calls on one
+    device must not overlap."""
     _check(lib().kvm_score_static(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(scores), _stream(stream)),
            "kvm_score_static")
 

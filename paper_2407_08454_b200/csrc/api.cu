@@ -44,9 +44,13 @@ int derive(const kvm_params* p, Dims& d) {
     return KVM_OK;
 }
 
+inline size_t score_row_bytes(const Dims& d) {
+    return d.dtype == KVM_BF16 ? score_tc_scratch_bytes_per_row() : sizeof(float);
+}
+
 struct Workspace {
     int* counters;      // 64 ints
-    float* lse;         // [B,Hq,S]
+    float* lse;         // row-pass output: [B,Hq,S] fp32 (fp32 path) or [B,Hq,S,16] bf16 side tensor (bf16 path)
     float* scores;      // [U,S]
     float* sim;         // [U,S]
     int32_t* set_start; // [U,cap+1]
@@ -60,7 +64,7 @@ Workspace carve(const Dims& d, void* base) {
     size_t off = 0;
     auto take = [&](size_t n) { size_t o = off; off += align_up(n); return (char*)base + o; };
     w.counters = (int*)take(64 * sizeof(int));
-    w.lse = (float*)take((size_t)d.B * d.Hq * d.S * sizeof(float));
+    w.lse = (float*)take((size_t)d.B * d.Hq * d.S * score_row_bytes(d));
     w.scores = (float*)take((size_t)d.U * d.S * sizeof(float));
     w.sim = (float*)take((size_t)d.U * d.S * sizeof(float));
     w.set_start = (int32_t*)take((size_t)d.U * (d.cap + 1) * sizeof(int32_t));
@@ -109,7 +113,7 @@ const char* kvm_status_string(int s) {
         case KVM_E_CUDA: return "CUDA runtime error";
         case KVM_E_DEVICE_TIMEOUT: return "a bounded device-side wait gave up";
         case KVM_E_STATIC_LIMIT:
-            return "batch * n_q_heads * seq exceeds the built-in scratch of kvm_score_static (KVM_STATIC_SCORE_ROWS)";
+            return "batch * n_q_heads * seq exceeds the built-in scratch of kvm_score_static (KVM_STATIC_SCORE_ROWS rows in fp32, an eighth of that in bf16)";
         default: return "unknown status";
     }
 }
@@ -289,7 +293,9 @@ int kvm_score_static(const kvm_params* p, const void* Q, const void* K, float* s
     if (rc != KVM_OK) return rc;
     if (!Q || !K || !scores) return KVM_E_NULL;
     if (misaligned(Q) || misaligned(K) || misaligned(scores)) return KVM_E_ALIGN;
-    if ((long long)d.B * d.Hq * d.S > (long long)KVM_STATIC_SCORE_ROWS) return KVM_E_STATIC_LIMIT;
+    // the row pass leaves 4 bytes per query row for fp32 tensors and 32 bytes for bf16 ones
+    if ((unsigned long long)d.B * d.Hq * d.S * score_row_bytes(d) > (unsigned long long)KVM_STATIC_SCORE_ROWS * sizeof(float))
+        return KVM_E_STATIC_LIMIT;
     unsigned char* base = (unsigned char*)static_scratch_for_current_device();
     if (!base) return KVM_E_CUDA;
     cudaStream_t st = (cudaStream_t)cuda_stream;

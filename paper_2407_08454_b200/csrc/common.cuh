@@ -54,6 +54,7 @@ cudaError_t launch_score_simt(const Dims& d, const void* Q, const void* K, const
                               float* scores, cudaStream_t st);
 cudaError_t launch_score_tc(const Dims& d, const void* Q, const void* K, const float* lse_in, float* lse_ws,
                             float* scores, kvm_stats* stats, cudaStream_t st);
+size_t score_tc_scratch_bytes_per_row();
 cudaError_t launch_similarity(const Dims& d, const void* K, float* sim, cudaStream_t st);
 cudaError_t launch_segment(const Dims& d, const float* scores, const float* sim, int32_t* set_id,
                            int32_t* set_start, int32_t* pivot, int32_t* out_len, kvm_stats* stats, cudaStream_t st);

@@ -14,6 +14,13 @@
 // transposed (A = keys), so a thread owns a key and adds up its column of the
 // attention map in registers, with no cross-lane reduction.
 //
+// Pass 2 needs exp(c s_ij - lse_i) with lse varying along the accumulator's columns.  Instead of
+// fetching lse per column in the epilogue, pass 1 stores e_i = -lse_i / c as three bf16 terms
+// (hi + mid + lo, 24 significant bits) in a 16-channel side tensor, and pass 2 appends one more
+// K = 16 MMA per step: A' = ones in the three channels, B' = that side tensor.  The tensor core,
+// which is far from busy here, then delivers q.k - lse/c directly and the epilogue is a bare
+// multiply, exponential and add per logit.
+//
 // One CTA per SM, persistent, warp-specialised:
 //   warps 0-15 epilogue: two groups of 8 take alternate steps; a warp reads TMEM lanes
 //              32*(w%4).. and one column half, does exp2 on the SFUs, keeps row/column state
@@ -39,6 +46,8 @@ constexpr int KCHUNK = 64;           // bf16 elements per 128-byte swizzle row
 constexpr int NSTAGE = 2;            // ring of B pairs (two 128-row tiles each)
 constexpr int NACC = 2;              // TMEM accumulator ring (2 x 256 columns = all 512)
 constexpr int ACC_COLS = 2 * TILE;   // accumulator columns per step
+constexpr int PCH = 16;              // channels of the lse side tensor (one K = 16 MMA slice; 3 are used)
+constexpr uint32_t PTILE_BYTES = TILE * PCH * 2;   // 4 KB: 128 rows x 32 B
 constexpr int NEPI_WARPS = 16;          // 4 TMEM lane quarters x 4 column quarters
 constexpr int QCOLS = TILE / 4;          // accumulator columns per epilogue warp
 constexpr int NTHREADS = (NEPI_WARPS + 2) * 32;
@@ -157,6 +166,11 @@ __device__ __forceinline__ uint64_t fadd2(uint64_t a, uint64_t b) {
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
     return r;
 }
+__device__ __forceinline__ uint64_t fmul2(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
 __device__ __forceinline__ uint64_t fsub2(uint64_t a, uint64_t b) {
     uint64_t r;
     asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
@@ -220,6 +234,16 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
     d |= (uint64_t)2 << 61;                         // 128-byte swizzle
     return d;
 }
+// Same for a tile of 32-byte rows (16 bf16 channels) with 32-byte swizzle: 8-row groups 256 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw32(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)(256u >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)6 << 61;                         // 32-byte swizzle
+    return d;
+}
 // kind::f16 instruction descriptor: fp32 accumulate, bf16 A and B, both K-major, M = 128, N = 128 or 256.
 constexpr uint32_t idesc_for(int n) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(TILE >> 4) << 24);
@@ -279,15 +303,14 @@ struct alignas(16) Shared {
     int abort_flag;
     float part_m[2][3][TILE];    // row states of warp sets 1..3 at item end, double-buffered by item parity
     float part_l[2][3][TILE];
-    alignas(16) float nlse_s[NEPI_WARPS][2][128];     // pass 2: each warp's own copy of -lse*log2(e) of its 64
-                                                      // columns of both sub-tiles of a step, double-buffered
 };
 
 template <int KCH>
 __global__ void __launch_bounds__(NTHREADS, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                const float* __restrict__ lse_in, float* __restrict__ lse_out, float* __restrict__ scores,
-                kvm_stats* stats, int pass, int B, int Hq, int Hkv, int S, float scale2) {
+                const __grid_constant__ CUtensorMap map_p, __nv_bfloat16* __restrict__ lsep_out,
+                float* __restrict__ scores, kvm_stats* stats, int pass, int B, int Hq, int Hkv, int S,
+                float scale2) {
     extern __shared__ uint8_t smem_raw[];
     constexpr uint32_t CHUNK_BYTES = TILE * 128;            // one [128 rows x 64 bf16] TMA box
     constexpr uint32_t TILE_BYTES = KCH * CHUNK_BYTES;      // an A tile: [KCH][128 rows][128 B]
@@ -297,7 +320,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     uint8_t* aligned = smem_raw + (base - smem_u32(smem_raw));
     uint8_t* sA = aligned;                                  // 2 A tiles
     uint8_t* sB = aligned + 2 * TILE_BYTES;                 // NSTAGE B pairs
-    Shared& sh = *reinterpret_cast<Shared*>(aligned + 2 * TILE_BYTES + NSTAGE * PAIR_BYTES);
+    uint8_t* sP = sB + NSTAGE * PAIR_BYTES;                 // NSTAGE pairs of lse side tiles (pass 2)
+    uint8_t* sOnes = sP + NSTAGE * 2 * PTILE_BYTES;         // constant A' tile: ones in the used channels
+    Shared& sh = *reinterpret_cast<Shared*>(sOnes + PTILE_BYTES);
     volatile int* abort_flag = &sh.abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -311,6 +336,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         for (int i = 0; i < NACC; ++i) { mbar_init(&sh.bar.acc_full[i], 1); mbar_init(&sh.bar.acc_empty[i], NEPI_WARPS / 2); }
         sh.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (pass == 2 && threadIdx.x < PTILE_BYTES / 16) {
+        // every 16-byte chunk of every row = bf16 {1, 1, 1, 0, 0, 0, 0, 0}: the same under any swizzle; the B'
+        // side tensor is zero outside channels 0..2, so the ones of the second chunk multiply zeros
+        reinterpret_cast<uint4*>(sOnes)[threadIdx.x] = make_uint4(0x3F803F80u, 0x00003F80u, 0u, 0u);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // visible to the tensor core's reads
     }
     if (warp == NEPI_WARPS + 1) tmem_alloc(&sh.tmem_base, NACC * ACC_COLS);
     tc_fence_before();
@@ -350,12 +381,15 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     ok = mbar_wait(&sh.bar.empty_b[s], ((cnt / NSTAGE) & 1) ^ 1, abort_flag);
                     if (!ok) break;
                     last_b[s] = (cnt / NSTAGE) & 1;
-                    mbar_expect_tx(&sh.bar.full_b[s], nh * TILE_BYTES);
+                    mbar_expect_tx(&sh.bar.full_b[s], nh * (TILE_BYTES + (pass == 2 ? PTILE_BYTES : 0u)));
                     for (int h = 0; h < nh; ++h) {
 #pragma unroll
                         for (int kc = 0; kc < KCH; ++kc)
                             tma_load_3d(sB + s * PAIR_BYTES + kc * PAIR_CHUNK + h * CHUNK_BYTES, mapB,
                                         &sh.bar.full_b[s], kc * KCHUNK, btile * TILE, bhead);
+                        if (pass == 2)
+                            tma_load_3d(sP + (s * 2 + h) * PTILE_BYTES, &map_p, &sh.bar.full_b[s], 0, btile * TILE,
+                                        bhead);
                         if (++btile == T && pass == 2) { btile = tile; ++bhead; }   // next query head of the group
                     }
                 }
@@ -380,6 +414,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             // descriptors differ from a buffer's first one only in the 16-byte-unit start address
             const uint64_t desc_a[2] = {smem_desc(base), smem_desc(base + TILE_BYTES)};
             const uint64_t desc_b0 = smem_desc(base + 2 * TILE_BYTES);
+            const uint64_t desc_p0 = smem_desc_sw32(base + 2 * TILE_BYTES + NSTAGE * PAIR_BYTES);
+            const uint64_t desc_ones = smem_desc_sw32(base + 2 * TILE_BYTES + NSTAGE * PAIR_BYTES + NSTAGE * 2 * PTILE_BYTES);
             for (int n = 0; ok && sc.item(n, head, tile); ++n) {
                 const int ab = n & 1;
                 ok = mbar_wait(&sh.bar.full_a[ab], (n >> 1) & 1, abort_flag);
@@ -400,6 +436,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         for (int ks = 0; ks < KCHUNK / 16; ++ks)
                             umma_bf16(d, da + ((kc * CHUNK_BYTES + ks * 32) >> 4), db + ((kc * PAIR_CHUNK + ks * 32) >> 4),
                                       idesc, (kc | ks) ? 1u : 0u);
+                    if (pass == 2)                         // + ones x (-lse/c): one more K = 16 slice
+                        umma_bf16(d, desc_ones, desc_p0 + (uint64_t)s * ((2 * PTILE_BYTES) >> 4), idesc, 1u);
                     umma_commit(&sh.bar.empty_b[s]);       // B stage reusable once these MMAs retire
                     umma_commit(&sh.bar.acc_full[as]);     // accumulator ready for the epilogue
                 }
@@ -422,27 +460,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         bool ok = true;
         StepIter it;
         it.init(sc);
-        // pass 2: the row-lse values of this warp's 64 columns are fetched one own-step ahead (lane c holds
-        // columns c and c + 32 of its half, for both sub-tiles of the step) and staged per warp
-        float lse_nx[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
-        auto fetch_step = [&](const StepIter& w) {
-            int g = w.bg, q = w.bt;
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const float* lse_h = lse_in + ((size_t)(w.head / Hkv) * Hq + (w.head % Hkv) * G + g) * S;
-                const int i0 = q * TILE + chalf * 64 + lane;
-                const bool live = w.valid && (w.t0 + h < w.nt);
-                // raw values; +inf (staged as -inf) zeroes columns past the sequence end
-                lse_nx[h][0] = (live && i0 < S) ? __ldg(lse_h + i0) : INFINITY;
-                lse_nx[h][1] = (live && i0 + 32 < S) ? __ldg(lse_h + i0 + 32) : INFINITY;
-                if (++q == T) { q = w.tile; ++g; }
-            }
-        };
-        if (pass == 2) {
-            StepIter la = it;
-            if (grp == 1) la.next(sc);
-            fetch_step(la);
-        }
         uint32_t own = 0;                                    // own steps processed (accumulator phase, staging parity)
         while (it.valid) {
             const int n = it.n, head = it.head, tile = it.tile;
@@ -451,20 +468,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             for (; it.valid && it.n == n; it.next(sc)) {
                 if ((int)(it.cnt & 1u) != grp) continue;
                 const int nh = (it.t0 + 1 < it.nt) ? 2 : 1;
-                if (pass == 2) {
-                    // stage this step's values (scaled to -lse*log2 e), then start the loads for the next own step
-                    float* stg = sh.nlse_s[warp][own & 1];
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        stg[h * 64 + lane] = lse_nx[h][0] * -LOG2E;
-                        stg[h * 64 + 32 + lane] = lse_nx[h][1] * -LOG2E;
-                    }
-                    StepIter la = it;
-                    la.next(sc);
-                    la.next(sc);
-                    fetch_step(la);
-                    __syncwarp();
-                }
                 ok = mbar_wait(&sh.bar.acc_full[grp], own & 1, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
                 if (ok) tc_fence_after();
@@ -517,23 +520,19 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                                 m = mnew;
                             }
                         } else {
-                            const uint64_t* nl =
-                                reinterpret_cast<const uint64_t*>(sh.nlse_s[warp][own & 1] + h * 64 + k * QCOLS);
-                            if (mask) {
+                            // The accumulator already holds q.k - lse/c: mask, scale, exponentiate, add.
+                            const int ncol = S - btile * TILE - cq * QCOLS;   // live columns of this chunk (queries < S)
+                            if (mask || ncol < QCOLS) {
 #pragma unroll
                                 for (int c = 0; c < QCOLS; ++c)
-                                    if (c < lane) v[c] = -INFINITY;      // query before key
+                                    if ((mask && c < lane) || c >= ncol) v[c] = -INFINITY;   // query before key, or past the end
                             }
 #pragma unroll
-                            for (int c = 0; c < QCOLS; c += 4) {
-                                const ulonglong2 n4 = *reinterpret_cast<const ulonglong2*>(nl + (c >> 1));
-                                float e0, e1, e2, e3;
-                                unpack2(ex2_pair(ffma2(pack2(v[c], v[c + 1]), sc2, n4.x), c >> 1), e0, e1);
-                                unpack2(ex2_pair(ffma2(pack2(v[c + 2], v[c + 3]), sc2, n4.y), (c >> 1) + 1), e2, e3);
+                            for (int c = 0; c < QCOLS; c += 2) {
+                                float e0, e1;
+                                unpack2(ex2_pair(fmul2(pack2(v[c], v[c + 1]), sc2), c >> 1), e0, e1);
                                 acc[c & 7] += e0;
                                 acc[(c + 1) & 7] += e1;
-                                acc[(c + 2) & 7] += e2;
-                                acc[(c + 3) & 7] += e3;
                             }
                         }
                     }
@@ -560,7 +559,16 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                             const float mq = sh.part_m[slot][q][row], lq_ = sh.part_l[slot][q][row];
                             if (mq > -INFINITY) L += lq_ * ex2(mq - M);
                         }
-                        lse_out[(size_t)head * S + gi] = bad ? NAN : (M + log2f(L)) * LN2;
+                        // e = -lse / c in the accumulator's units (lse in log2 units is M + log2 L), as hi + mid + lo
+                        const float e = bad ? NAN : -(M + log2f(L)) / scale2;
+                        const __nv_bfloat16 eh = __float2bfloat16_rn(e);
+                        const float r1 = e - __bfloat162float(eh);
+                        const __nv_bfloat16 em = __float2bfloat16_rn(r1);
+                        const __nv_bfloat16 el = __float2bfloat16_rn(r1 - __bfloat162float(em));
+                        uint4* dst = reinterpret_cast<uint4*>(lsep_out + ((size_t)head * S + gi) * PCH);
+                        dst[0] = make_uint4((uint32_t)__bfloat16_as_ushort(eh) | ((uint32_t)__bfloat16_as_ushort(em) << 16),
+                                            (uint32_t)__bfloat16_as_ushort(el), 0u, 0u);
+                        dst[1] = make_uint4(0u, 0u, 0u, 0u);
                     } else {
                         const float tot = (mine + sh.part_l[slot][0][row]) + (sh.part_l[slot][1][row] + sh.part_l[slot][2][row]);
                         scores[(size_t)head * S + gi] = bad ? NAN : tot / (float)G;
@@ -607,10 +615,40 @@ bool make_map(CUtensorMap* map, const void* ptr, int heads, int S, int D) {
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// [heads, S, 16] bf16 side tensor of pass 2: boxes of [1, 128 rows, 16 channels] (32-byte rows), 32-byte swizzle.
+bool make_map_side(CUtensorMap* map, const void* ptr, int heads, int S) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)PCH, (cuuint64_t)S, (cuuint64_t)heads};
+    cuuint64_t strides[2] = {(cuuint64_t)PCH * 2, (cuuint64_t)S * PCH * 2};
+    cuuint32_t box[3] = {PCH, TILE, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Caller-supplied natural-log lse -> the side tensor pass 2 multiplies in (e = -lse * log2(e) / scale2 as hi+mid+lo).
+__global__ void __launch_bounds__(256) lse_split_kernel(const float* __restrict__ lse, __nv_bfloat16* __restrict__ side,
+                                                        long long rows, float neg_log2e_over_scale2) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= rows) return;
+    const float e = lse[i] * neg_log2e_over_scale2;
+    const __nv_bfloat16 eh = __float2bfloat16_rn(e);
+    const float r1 = e - __bfloat162float(eh);
+    const __nv_bfloat16 em = __float2bfloat16_rn(r1);
+    const __nv_bfloat16 el = __float2bfloat16_rn(r1 - __bfloat162float(em));
+    uint4* dst = reinterpret_cast<uint4*>(side + (size_t)i * PCH);
+    dst[0] = make_uint4((uint32_t)__bfloat16_as_ushort(eh) | ((uint32_t)__bfloat16_as_ushort(em) << 16),
+                        (uint32_t)__bfloat16_as_ushort(el), 0u, 0u);
+    dst[1] = make_uint4(0u, 0u, 0u, 0u);
+}
+
 template <int KCH>
-cudaError_t launch_t(const Dims& d, const CUtensorMap& mq, const CUtensorMap& mk, const float* lse_in, float* lse_ws,
-                     float* scores, kvm_stats* stats, cudaStream_t st) {
-    const size_t smem = 1024 + (size_t)(2 + 2 * NSTAGE) * KCH * TILE * 128 + sizeof(Shared);
+cudaError_t launch_t(const Dims& d, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mp,
+                     const float* lse_in, __nv_bfloat16* side, float* scores, kvm_stats* stats, cudaStream_t st) {
+    const size_t smem = 1024 + (size_t)(2 + 2 * NSTAGE) * KCH * TILE * 128 + (size_t)(2 * NSTAGE + 1) * PTILE_BYTES +
+                        sizeof(Shared);
     cudaError_t e = cudaFuncSetAttribute(score_tc_kernel<KCH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     int dev = 0, sms = 0;
@@ -618,31 +656,37 @@ cudaError_t launch_t(const Dims& d, const CUtensorMap& mq, const CUtensorMap& mk
     if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
     const int T = (d.S + TILE - 1) / TILE;
     const float scale2 = d.scale * LOG2E;
-    const float* lse = lse_in;
     if (!lse_in) {
         const long long items = (long long)d.B * d.Hq * T;
         const int grid = (int)(items < sms ? items : sms);
-        score_tc_kernel<KCH><<<grid, NTHREADS, smem, st>>>(mq, mk, nullptr, lse_ws, nullptr, stats, 1, d.B, d.Hq,
-                                                          d.Hkv, d.S, scale2);
-        if ((e = cudaGetLastError()) != cudaSuccess) return e;
-        lse = lse_ws;
+        score_tc_kernel<KCH><<<grid, NTHREADS, smem, st>>>(mq, mk, mp, side, nullptr, stats, 1, d.B, d.Hq, d.Hkv, d.S,
+                                                          scale2);
+    } else {
+        const long long rows = (long long)d.B * d.Hq * d.S;
+        lse_split_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(lse_in, side, rows, -LOG2E / scale2);
     }
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
     const long long items = (long long)d.U * T;
     const int grid = (int)(items < sms ? items : sms);
-    score_tc_kernel<KCH><<<grid, NTHREADS, smem, st>>>(mq, mk, lse, nullptr, scores, stats, 2, d.B, d.Hq, d.Hkv, d.S,
+    score_tc_kernel<KCH><<<grid, NTHREADS, smem, st>>>(mq, mk, mp, nullptr, scores, stats, 2, d.B, d.Hq, d.Hkv, d.S,
                                                       scale2);
     return cudaGetLastError();
 }
 
 }  // namespace
 
+// Bytes of scratch per query row that the tensor-core path needs (the lse side tensor).
+size_t score_tc_scratch_bytes_per_row() { return (size_t)PCH * 2; }
+
 cudaError_t launch_score_tc(const Dims& d, const void* Q, const void* K, const float* lse_in, float* lse_ws,
                             float* scores, kvm_stats* stats, cudaStream_t st) {
-    CUtensorMap mq, mk;
-    if (!make_map(&mq, Q, d.B * d.Hq, d.S, d.D) || !make_map(&mk, K, d.B * d.Hkv, d.S, d.D))
+    CUtensorMap mq, mk, mp;
+    __nv_bfloat16* side = reinterpret_cast<__nv_bfloat16*>(lse_ws);
+    if (!make_map(&mq, Q, d.B * d.Hq, d.S, d.D) || !make_map(&mk, K, d.B * d.Hkv, d.S, d.D) ||
+        !make_map_side(&mp, side, d.B * d.Hq, d.S))
         return cudaErrorNotSupported;
-    return d.D == 128 ? launch_t<2>(d, mq, mk, lse_in, lse_ws, scores, stats, st)
-                      : launch_t<1>(d, mq, mk, lse_in, lse_ws, scores, stats, st);
+    return d.D == 128 ? launch_t<2>(d, mq, mk, mp, lse_in, side, scores, stats, st)
+                      : launch_t<1>(d, mq, mk, mp, lse_in, side, scores, stats, st);
 }
 
 }  // namespace kvm
