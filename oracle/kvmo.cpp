@@ -213,11 +213,23 @@ void kvmo_pivots(int64_t U, int32_t S, int32_t cap, const double* scores,
     }
 }
 
+// Pivot of the average-weighted baseline (Section 4.2, first experiment): the
+// state with the maximum index within each merging set.
+void kvmo_pivots_last(int64_t U, int32_t cap, const int32_t* set_start, const int32_t* out_len, int32_t* pivot) {
+    for (int64_t u = 0; u < U; ++u) {
+        const int32_t* st = set_start + (size_t)u * (cap + 1);
+        for (int32_t s = 0; s < out_len[u]; ++s) pivot[(size_t)u * cap + s] = st[s + 1] - 1;
+    }
+}
+
 // Algorithm 2, weights and merge (Eq. 4, Eq. 5, Definition 4.2), fixed sigma:
 //   g_j = exp(-|k_p - k_j|^2 / (2 sigma^2)),  w_j = g_j / sum_{t in set} g_t   (g_p = 1)
 //   K*_s = sum_j w_j k_j;   V*_s = (|set| if scale_v else 1) * sum_j w_j v_j
+// weight_rule 0 is the paper's method.  1 = average-weighted merging (Section
+// 4.2's baseline): g_j = 1, so w_j = 1/|set|.  2 = the sigma -> 0 limit named
+// after Eq. 5: nothing but the pivot survives, g_j = [j == p].
 // K_out, V_out [U,cap,D] fp64 (rows >= out_len untouched); weights (nullable) [U,S].
-void kvmo_merge(int64_t U, int32_t S, int32_t D, int32_t cap, double sigma, int32_t scale_v,
+void kvmo_merge(int64_t U, int32_t S, int32_t D, int32_t cap, double sigma, int32_t scale_v, int32_t weight_rule,
                 const float* K, const float* V, const int32_t* set_start, const int32_t* pivot,
                 const int32_t* out_len, double* K_out, double* V_out, double* weights) {
 #pragma omp parallel for schedule(dynamic)
@@ -237,7 +249,9 @@ void kvmo_merge(int64_t U, int32_t S, int32_t D, int32_t cap, double sigma, int3
                     const double df = (double)kp[t] - (double)kj[t];
                     d2 += df * df;
                 }
-                g[j] = std::exp(-d2 / (2.0 * sigma * sigma));
+                if (weight_rule == 1) g[j] = 1.0;
+                else if (weight_rule == 2) g[j] = (j == p) ? 1.0 : 0.0;
+                else g[j] = std::exp(-d2 / (2.0 * sigma * sigma));
                 gsum += g[j];
             }
             double* ko = K_out + ((size_t)u * cap + s) * D;
@@ -258,11 +272,40 @@ void kvmo_merge(int64_t U, int32_t S, int32_t D, int32_t cap, double sigma, int3
     }
 }
 
+// Eviction for comparison (Section 2.2; the heavy-hitter scheme the paper
+// measures against in Section 4.2 and Section 5): only the conserved tokens --
+// the n_h largest aggregated scores and the n_r most recent -- stay, unchanged
+// and in token order; everything else is dropped.  out_pos [U,cap] = the kept
+// token indices; K_out, V_out [U,cap,D]; out_len [U] = number kept (<= cap required).
+void kvmo_evict(int64_t U, int32_t S, int32_t D, int32_t cap, const uint8_t* keep, const float* K, const float* V,
+                int32_t* out_len, int32_t* out_pos, double* K_out, double* V_out) {
+    for (int64_t u = 0; u < U; ++u) {
+        int32_t n = 0;
+        for (int32_t j = 0; j < S; ++j) {
+            if (!keep[(size_t)u * S + j]) continue;
+            if (n < cap) {
+                out_pos[(size_t)u * cap + n] = j;
+                for (int32_t t = 0; t < D; ++t) {
+                    K_out[((size_t)u * cap + n) * D + t] = (double)K[((size_t)u * S + j) * D + t];
+                    V_out[((size_t)u * cap + n) * D + t] = (double)V[((size_t)u * S + j) * D + t];
+                }
+            }
+            ++n;
+        }
+        out_len[u] = n;
+    }
+}
+
 // The whole path for one layer, steps in the paper's order.  All outputs are
 // caller-allocated; cap = C when enforce_budget, else S.
+// Variants (all 0 = the paper's method): pivot_rule 1 = last index of the set,
+// 2 = arg-max of pivot_key [U,S] (iid random numbers give the random-pivot
+// ablation of Section 5.3); weight_rule as in kvmo_merge; set_rule 1 = eviction
+// (kvmo_evict; set_id is -1 for dropped tokens, set_start[s] = the kept token).
 void kvmo_compress(int32_t B, int32_t Hq, int32_t Hkv, int32_t S, int32_t D, double scale,
                    int32_t cap, int32_t n_r, int32_t n_h, double eps, double sigma,
                    int32_t scale_v, int32_t enforce_budget,
+                   int32_t pivot_rule, int32_t weight_rule, int32_t set_rule, const double* pivot_key,
                    const float* Q, const float* K, const float* V,
                    double* scores, uint8_t* keep, double* sim, uint8_t* b,
                    int32_t* set_id, int32_t* set_start, int32_t* out_len, int32_t* pivot,
@@ -271,10 +314,26 @@ void kvmo_compress(int32_t B, int32_t Hq, int32_t Hkv, int32_t S, int32_t D, dou
     kvmo_scores(B, Hq, Hkv, S, D, scale, Q, K, scores, nullptr);
     kvmo_keep(U, S, n_r, n_h, scores, keep);
     kvmo_similarity(U, S, D, K, sim);
+    if (set_rule == 1) {
+        kvmo_evict(U, S, D, cap, keep, K, V, out_len, pivot, K_out, V_out);
+        for (int64_t u = 0; u < U; ++u) {
+            int32_t n = 0;
+            for (int32_t j = 0; j < S; ++j) {
+                const bool k = keep[(size_t)u * S + j] != 0;
+                b[(size_t)u * S + j] = k;
+                set_id[(size_t)u * S + j] = k ? n : -1;
+                if (k && n <= cap) set_start[(size_t)u * (cap + 1) + n] = j;
+                n += k;
+            }
+            if (n <= cap) set_start[(size_t)u * (cap + 1) + n] = S;
+        }
+        return;
+    }
     kvmo_boundaries(U, S, cap, eps, enforce_budget, sim, keep, b, nullptr);
     kvmo_sets(U, S, cap, b, set_id, set_start, out_len);
-    kvmo_pivots(U, S, cap, scores, set_start, out_len, pivot);
-    kvmo_merge(U, S, D, cap, sigma, scale_v, K, V, set_start, pivot, out_len, K_out, V_out, nullptr);
+    if (pivot_rule == 1) kvmo_pivots_last(U, cap, set_start, out_len, pivot);
+    else kvmo_pivots(U, S, cap, pivot_rule == 2 ? pivot_key : scores, set_start, out_len, pivot);
+    kvmo_merge(U, S, D, cap, sigma, scale_v, weight_rule, K, V, set_start, pivot, out_len, K_out, V_out, nullptr);
 }
 
 }  // extern "C"

@@ -128,7 +128,38 @@ def pivots(scores_: np.ndarray, set_start: np.ndarray, out_len: np.ndarray) -> n
     return pv
 
 
-def merge(K, V, set_start, pivot, out_len, sigma: float, scale_v: bool = True, want_weights: bool = False):
+def pivots_last(set_start: np.ndarray, out_len: np.ndarray) -> np.ndarray:
+    set_start = np.ascontiguousarray(set_start, dtype=np.int32)
+    out_len = np.ascontiguousarray(out_len, dtype=np.int32)
+    cap = set_start.shape[-1] - 1
+    U = out_len.size
+    pv = np.full(out_len.shape + (cap,), -1, dtype=np.int32)
+    lib().kvmo_pivots_last(ctypes.c_int64(U), ctypes.c_int32(cap), _p(set_start), _p(out_len), _p(pv))
+    return pv
+
+
+def evict(keep_: np.ndarray, K, V, cap: int):
+    K, V = _f32(K), _f32(V)
+    keep_ = np.ascontiguousarray(keep_, dtype=np.uint8)
+    S, D = K.shape[-2:]
+    U = K.size // (S * D)
+    lead = K.shape[:-2]
+    out_len = np.empty(lead, np.int32)
+    out_pos = np.full(lead + (cap,), -1, np.int32)
+    Ko = np.full(lead + (cap, D), np.nan, dtype=np.float64)
+    Vo = np.full(lead + (cap, D), np.nan, dtype=np.float64)
+    lib().kvmo_evict(ctypes.c_int64(U), ctypes.c_int32(S), ctypes.c_int32(D), ctypes.c_int32(cap), _p(keep_),
+                     _p(K), _p(V), _p(out_len), _p(out_pos), _p(Ko), _p(Vo))
+    return out_len, out_pos, Ko, Vo
+
+
+PIVOT_MAX_SCORE, PIVOT_LAST, PIVOT_KEY = 0, 1, 2
+WEIGHT_GAUSSIAN, WEIGHT_AVERAGE, WEIGHT_PIVOT_ONLY = 0, 1, 2
+SETS_ADJACENT, SETS_CONSERVED_ONLY = 0, 1
+
+
+def merge(K, V, set_start, pivot, out_len, sigma: float, scale_v: bool = True, want_weights: bool = False,
+          weight_rule: int = 0):
     K, V = _f32(K), _f32(V)
     set_start = np.ascontiguousarray(set_start, dtype=np.int32)
     pivot = np.ascontiguousarray(pivot, dtype=np.int32)
@@ -141,7 +172,8 @@ def merge(K, V, set_start, pivot, out_len, sigma: float, scale_v: bool = True, w
     Vo = np.full(lead + (cap, D), np.nan, dtype=np.float64)
     w = np.full(lead + (S,), np.nan, dtype=np.float64) if want_weights else None
     lib().kvmo_merge(ctypes.c_int64(U), ctypes.c_int32(S), ctypes.c_int32(D), ctypes.c_int32(cap),
-                     ctypes.c_double(sigma), ctypes.c_int32(1 if scale_v else 0), _p(K), _p(V), _p(set_start),
+                     ctypes.c_double(sigma), ctypes.c_int32(1 if scale_v else 0), ctypes.c_int32(weight_rule),
+                     _p(K), _p(V), _p(set_start),
                      _p(pivot), _p(out_len), _p(Ko), _p(Vo), _p(w))
     return (Ko, Vo, w) if want_weights else (Ko, Vo)
 
@@ -164,7 +196,8 @@ class Compressed:
 
 
 def compress(Q, K, V, budget: float, recent: float, heavy: float, eps: float = 0.75, sigma: float = 5.0,
-             scale: Optional[float] = None, scale_v: bool = True, enforce_budget: bool = True) -> Compressed:
+             scale: Optional[float] = None, scale_v: bool = True, enforce_budget: bool = True,
+             pivot_rule: int = 0, weight_rule: int = 0, set_rule: int = 0, pivot_key=None) -> Compressed:
     """All steps for one layer through the single C entry point kvmo_compress."""
     Q, K, V = _f32(Q), _f32(K), _f32(V)
     B, Hq, S, D = Q.shape
@@ -174,6 +207,10 @@ def compress(Q, K, V, budget: float, recent: float, heavy: float, eps: float = 0
     C, n_r, n_h = sizes(S, budget, recent, heavy)
     cap = C if enforce_budget else S
     lead = (B, Hkv)
+    if pivot_key is not None:
+        pivot_key = np.ascontiguousarray(pivot_key, dtype=np.float64)
+        assert pivot_key.shape == lead + (S,)
+    assert (pivot_rule == PIVOT_KEY) == (pivot_key is not None)
     r = Compressed(
         scores=np.empty(lead + (S,), np.float64), keep=np.empty(lead + (S,), np.uint8),
         sim=np.empty(lead + (S,), np.float64), b=np.empty(lead + (S,), np.uint8),
@@ -185,6 +222,7 @@ def compress(Q, K, V, budget: float, recent: float, heavy: float, eps: float = 0
                         ctypes.c_int32(D), ctypes.c_double(scale), ctypes.c_int32(cap), ctypes.c_int32(n_r),
                         ctypes.c_int32(n_h), ctypes.c_double(eps), ctypes.c_double(sigma),
                         ctypes.c_int32(1 if scale_v else 0), ctypes.c_int32(1 if enforce_budget else 0),
-                        _p(Q), _p(K), _p(V), _p(r.scores), _p(r.keep), _p(r.sim), _p(r.b), _p(r.set_id),
+                        ctypes.c_int32(pivot_rule), ctypes.c_int32(weight_rule), ctypes.c_int32(set_rule),
+                        _p(pivot_key), _p(Q), _p(K), _p(V), _p(r.scores), _p(r.keep), _p(r.sim), _p(r.b), _p(r.set_id),
                         _p(r.set_start), _p(r.out_len), _p(r.pivot), _p(r.K_out), _p(r.V_out))
     return r

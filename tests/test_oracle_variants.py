@@ -1,0 +1,144 @@
+"""Pins for the CPU checker's variants of the method: the average-weighted
+baseline with last-index pivots (Section 4.2), pivots by a caller-supplied key
+(the random-pivot ablation of Section 5.3), the pivot-only limit named after
+Eq. 5, and eviction of everything but the conserved tokens (Section 2.2).
+Library routines, limits of the pinned Gaussian merge, and invariants only."""
+import numpy as np
+import pytest
+
+from oracle import kvmo
+from paper_2407_08454_b200 import synth_inputs as si
+
+
+def _rand(shape, seed):
+    return np.random.default_rng(seed).standard_normal(shape).astype(np.float32)
+
+
+def _random_partition(S, U, seed, p=0.3):
+    b = (np.random.default_rng(seed).random((U, S)) < p).astype(np.uint8)
+    b[:, 0] = 1
+    return kvmo.sets(b, cap=S)
+
+
+def test_last_index_pivot_is_the_set_maximum_index():
+    set_id, st, ol = _random_partition(80, 3, 0)
+    pv = kvmo.pivots_last(st, ol)
+    for u in range(3):
+        for s in range(ol[u]):
+            members = np.nonzero(set_id[u] == s)[0]
+            assert pv[u, s] == members.max()
+        assert (pv[u, ol[u]:] == -1).all()
+    # same thing as an arg-max whose key grows with the index
+    np.testing.assert_array_equal(pv, kvmo.pivots(np.tile(np.arange(80.0), (3, 1)), st, ol))
+
+
+def test_key_pivot_is_uniform_over_the_set_for_iid_keys():
+    # one set of 5 tokens, many independent draws: every member is chosen about equally often
+    n, trials = 5, 4000
+    b = np.zeros((trials, n), np.uint8)
+    b[:, 0] = 1
+    _, st, ol = kvmo.sets(b, cap=n)
+    key = np.random.default_rng(1).random((trials, n))
+    pv = kvmo.pivots(key, st, ol)[:, 0]
+    np.testing.assert_array_equal(pv, key.argmax(1))
+    counts = np.bincount(pv, minlength=n)
+    chi2 = ((counts - trials / n) ** 2 / (trials / n)).sum()
+    assert chi2 < 18.5          # 99.9 % point of chi-square with 4 degrees of freedom
+
+
+def test_average_rule_is_the_library_mean():
+    K, V = _rand((2, 50, 6), 2), _rand((2, 50, 6), 3)
+    set_id, st, ol = _random_partition(50, 2, 4)
+    pv = kvmo.pivots_last(st, ol)
+    Ko, Vo, w = kvmo.merge(K, V, st, pv, ol, sigma=5.0, scale_v=False, want_weights=True,
+                           weight_rule=kvmo.WEIGHT_AVERAGE)
+    Ks, Vs, _ = kvmo.merge(K, V, st, pv, ol, sigma=5.0, scale_v=True, want_weights=True,
+                           weight_rule=kvmo.WEIGHT_AVERAGE)
+    for u in range(2):
+        for s in range(ol[u]):
+            m = set_id[u] == s
+            np.testing.assert_allclose(Ko[u, s], K[u, m].astype(np.float64).mean(0), rtol=1e-13, atol=1e-15)
+            np.testing.assert_allclose(Vo[u, s], V[u, m].astype(np.float64).mean(0), rtol=1e-13, atol=1e-15)
+            np.testing.assert_allclose(Vs[u, s], V[u, m].astype(np.float64).sum(0), rtol=1e-13, atol=1e-13)
+            np.testing.assert_allclose(w[u, m], 1.0 / m.sum(), rtol=1e-15)
+    np.testing.assert_array_equal(Ks[0, :ol[0]], Ko[0, :ol[0]])    # keys never carry the set size
+    # and it is the Gaussian rule's sigma -> infinity limit, whatever the pivot
+    Kg, Vg = kvmo.merge(K, V, st, kvmo.pivots(_rand((2, 50), 5), st, ol), ol, sigma=1e9, scale_v=False)
+    np.testing.assert_allclose(Kg[0, :ol[0]], Ko[0, :ol[0]], rtol=1e-12, atol=1e-14)
+
+
+def test_pivot_only_rule_copies_the_pivot_rows():
+    K, V = _rand((2, 40, 5), 6), _rand((2, 40, 5), 7)
+    set_id, st, ol = _random_partition(40, 2, 8)
+    pv = kvmo.pivots(_rand((2, 40), 9), st, ol)
+    Ko, Vo, w = kvmo.merge(K, V, st, pv, ol, sigma=5.0, scale_v=False, want_weights=True,
+                           weight_rule=kvmo.WEIGHT_PIVOT_ONLY)
+    for u in range(2):
+        n = ol[u]
+        np.testing.assert_array_equal(Ko[u, :n], K[u, pv[u, :n]].astype(np.float64))
+        np.testing.assert_array_equal(Vo[u, :n], V[u, pv[u, :n]].astype(np.float64))
+        assert w[u].sum() == n and set(np.unique(w[u])) <= {0.0, 1.0}
+    # the Gaussian rule tends to it as sigma -> 0 (distinct keys)
+    Kg, Vg = kvmo.merge(K, V, st, pv, ol, sigma=1e-3, scale_v=False)
+    np.testing.assert_allclose(Kg[0, :ol[0]], Ko[0, :ol[0]], rtol=1e-12)
+    # with the set-size factor the value row is the pivot's value times the set size
+    _, Vs = kvmo.merge(K, V, st, pv, ol, sigma=5.0, scale_v=True, weight_rule=kvmo.WEIGHT_PIVOT_ONLY)
+    sizes = np.diff(st[0, :ol[0] + 1])
+    np.testing.assert_array_equal(Vs[0, :ol[0]], Vo[0, :ol[0]] * sizes[:, None])
+
+
+def test_eviction_keeps_exactly_the_conserved_rows_in_order():
+    rng = np.random.default_rng(10)
+    K, V = _rand((3, 30, 4), 11), _rand((3, 30, 4), 12)
+    a = rng.random((3, 30))
+    keep = kvmo.keep(a, 6, 5)
+    ol, pos, Ko, Vo = kvmo.evict(keep, K, V, cap=11)
+    for u in range(3):
+        idx = np.nonzero(keep[u])[0]                       # numpy's own gather is the definition
+        assert ol[u] == len(idx) == 11
+        np.testing.assert_array_equal(pos[u], idx)
+        np.testing.assert_array_equal(Ko[u], K[u, idx].astype(np.float64))
+        np.testing.assert_array_equal(Vo[u], V[u, idx].astype(np.float64))
+        # heavy hitters: every kept non-recent score is at least every dropped score
+        old = idx[idx < 24]
+        dropped = np.setdiff1d(np.arange(24), old)
+        assert a[u, old].min() >= a[u, dropped].max()
+    # nothing conserved -> nothing kept; everything conserved -> the cache itself
+    ol, pos, Ko, Vo = kvmo.evict(np.zeros((1, 30), np.uint8), K[:1], V[:1], cap=4)
+    assert ol[0] == 0 and (pos == -1).all() and np.isnan(Ko).all()
+    ol, pos, Ko, Vo = kvmo.evict(np.ones((1, 30), np.uint8), K[:1], V[:1], cap=30)
+    np.testing.assert_array_equal(Ko[0], K[0].astype(np.float64))
+
+
+def test_compress_variants_equal_their_steps():
+    cfg = si.CONFIGS["C0"]
+    d = si.make_layer(cfg)
+    base = kvmo.compress(d["Q"], d["K"], d["V"], 0.50, 0.17, 0.12)
+    S, U = cfg.seq, cfg.n_kv_heads
+    key = np.random.default_rng(13).random((1, U, S))
+    # average-weighted baseline: same sets as the method, last-index pivots, plain means
+    r = kvmo.compress(d["Q"], d["K"], d["V"], 0.50, 0.17, 0.12, scale_v=False,
+                      pivot_rule=kvmo.PIVOT_LAST, weight_rule=kvmo.WEIGHT_AVERAGE)
+    np.testing.assert_array_equal(r.set_start, base.set_start)
+    np.testing.assert_array_equal(r.pivot, kvmo.pivots_last(base.set_start, base.out_len))
+    Ko, Vo = kvmo.merge(d["K"], d["V"], base.set_start, r.pivot, base.out_len, 5.0, scale_v=False,
+                        weight_rule=kvmo.WEIGHT_AVERAGE)
+    np.testing.assert_array_equal(r.K_out, Ko)
+    # keyed pivots: sets unchanged, conserved tokens still their own pivot, pivots differ somewhere
+    r = kvmo.compress(d["Q"], d["K"], d["V"], 0.50, 0.17, 0.12, pivot_rule=kvmo.PIVOT_KEY, pivot_key=key)
+    np.testing.assert_array_equal(r.set_start, base.set_start)
+    np.testing.assert_array_equal(r.pivot, kvmo.pivots(key, base.set_start, base.out_len))
+    assert (r.pivot != base.pivot).any()
+    for u in range(U):
+        kept = np.nonzero(base.keep[0, u])[0]
+        np.testing.assert_array_equal(r.pivot[0, u, base.set_id[0, u, kept]], kept)
+    # eviction with the heavy share filling the budget: exactly cap rows, all of them input rows
+    r = kvmo.compress(d["Q"], d["K"], d["V"], 0.50, 0.17, 0.50 - 0.17, set_rule=kvmo.SETS_CONSERVED_ONLY)
+    K64 = d["K"].double().numpy()
+    for u in range(U):
+        n = r.out_len[0, u]
+        assert n == r.n_r + r.n_h and n <= r.cap
+        idx = np.nonzero(r.keep[0, u])[0]
+        np.testing.assert_array_equal(r.pivot[0, u, :n], idx)
+        np.testing.assert_array_equal(r.K_out[0, u, :n], K64[0, u, idx])
+        assert (r.set_id[0, u, idx] == np.arange(n)).all() and (np.delete(r.set_id[0, u], idx) == -1).all()
