@@ -42,7 +42,7 @@
 extern "C" {
 #endif
 
-#define KVM_VERSION 100
+#define KVM_VERSION 101
 
 enum kvm_dtype { KVM_BF16 = 0, KVM_F32 = 1 };
 
@@ -51,7 +51,7 @@ enum kvm_status {
     KVM_E_NULL = -1,        /* a required pointer is NULL */
     KVM_E_SHAPE = -2,       /* sizes not positive, heads not divisible, head_dim not 64/128, seq too long */
     KVM_E_DTYPE = -3,       /* dtype is not a kvm_dtype */
-    KVM_E_PARAM = -4,       /* ratio/threshold/bandwidth out of range, or capacity too small for the conserved set */
+    KVM_E_PARAM = -4,       /* ratio/threshold/bandwidth/rule out of range, or capacity too small for the conserved set */
     KVM_E_ALIGN = -5,       /* a tensor pointer is not 16-byte aligned */
     KVM_E_WORKSPACE = -6,   /* ws is NULL or smaller than kvm_workspace_bytes() */
     KVM_E_UNSUPPORTED = -7, /* valid request this build cannot run (e.g. non-causal) */
@@ -73,7 +73,36 @@ typedef struct kvm_params {
     int32_t causal;              /* must be 1 */
     int32_t scale_v_by_set_size; /* 1: value weights are multiplied by the set size (text after Eq. 5); 0: plain weighted mean */
     int32_t enforce_budget;      /* 1: at most floor(budget*S) sets per unit (see kvm_segment); 0: capacity is S */
+    /* Variants the paper describes beside its method.  All zero = the method itself. */
+    int32_t pivot_rule;          /* kvm_pivot_rule */
+    int32_t weight_rule;         /* kvm_weight_rule */
+    int32_t set_rule;            /* kvm_set_rule */
+    const float* pivot_key;      /* device [U, S] fp32, finite; read only when pivot_rule == KVM_PIVOT_KEY, else NULL */
 } kvm_params;
+
+/* How the pivot of a merging set is chosen. */
+enum kvm_pivot_rule {
+    KVM_PIVOT_MAX_SCORE = 0, /* largest aggregated attention score (Eq. 6) */
+    KVM_PIVOT_LAST = 1,      /* the set's maximum token index (the average-weighted baseline of Section 4.2) */
+    KVM_PIVOT_KEY = 2        /* largest pivot_key, ties to the lowest index; iid random keys give the random-pivot
+                                ablation of Section 5.3.  The conserved set still comes from the attention scores. */
+};
+/* How a set's states are weighted. */
+enum kvm_weight_rule {
+    KVM_WEIGHT_GAUSSIAN = 0,  /* Eq. 4, Eq. 5 with the fixed sigma */
+    KVM_WEIGHT_AVERAGE = 1,   /* every state 1/|set| (average-weighted merging, Section 4.2); sigma is ignored */
+    KVM_WEIGHT_PIVOT_ONLY = 2 /* the sigma -> 0 limit noted after Eq. 5: the pivot's own K and V rows, nothing
+                                 merged in (V still times the set size when scale_v_by_set_size) */
+};
+/* Which states reach the output. */
+enum kvm_set_rule {
+    KVM_SETS_ADJACENT = 0,       /* Algorithm 1: every token belongs to a merging set */
+    KVM_SETS_CONSERVED_ONLY = 1  /* eviction as in the heavy-hitter schemes of Section 2.2: only the conserved tokens
+                                    (largest scores + most recent) stay, unchanged, in token order; pivot_rule,
+                                    weight_rule, sim_threshold and sigma are ignored, out_len = n_recent + n_heavy,
+                                    which must fit the capacity; set_id is -1 for dropped tokens and
+                                    set_start[s] = pivot[s] = the s-th kept token */
+};
 
 #define KVM_MAX_SEQ 65536
 

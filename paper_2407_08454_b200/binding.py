@@ -19,6 +19,9 @@ LIB_PATH = os.path.join(_PKG, "libkvm.so")
 
 KVM_BF16, KVM_F32 = 0, 1
 KVM_OK = 0
+KVM_PIVOT_MAX_SCORE, KVM_PIVOT_LAST, KVM_PIVOT_KEY = 0, 1, 2
+KVM_WEIGHT_GAUSSIAN, KVM_WEIGHT_AVERAGE, KVM_WEIGHT_PIVOT_ONLY = 0, 1, 2
+KVM_SETS_ADJACENT, KVM_SETS_CONSERVED_ONLY = 0, 1
 EXPORTS = (
     "kvm_sizes", "kvm_workspace_bytes", "kvm_score", "kvm_segment", "kvm_merge_compact", "kvm_compress",
     "kvm_host_staging_bytes", "kvm_compress_host", "kvm_score_static", "kvm_status_string", "kvm_version",
@@ -34,6 +37,8 @@ class KvmParams(ctypes.Structure):
         ("budget", ctypes.c_float), ("recent_ratio", ctypes.c_float), ("heavy_ratio", ctypes.c_float),
         ("sim_threshold", ctypes.c_float), ("sigma", ctypes.c_float), ("softmax_scale", ctypes.c_float),
         ("causal", ctypes.c_int32), ("scale_v_by_set_size", ctypes.c_int32), ("enforce_budget", ctypes.c_int32),
+        ("pivot_rule", ctypes.c_int32), ("weight_rule", ctypes.c_int32), ("set_rule", ctypes.c_int32),
+        ("pivot_key", ctypes.c_void_p),
     ]
 
 
@@ -79,11 +84,19 @@ def status_string(status: int) -> str:
 def make_params(batch: int, n_q_heads: int, n_kv_heads: int, seq: int, head_dim: int, dtype,
                 budget: float = 0.5, recent_ratio: float = -1.0, heavy_ratio: float = -1.0,
                 sim_threshold: float = 0.75, sigma: float = 5.0, softmax_scale: float = 0.0, causal: int = 1,
-                scale_v_by_set_size: int = 1, enforce_budget: int = 1) -> KvmParams:
+                scale_v_by_set_size: int = 1, enforce_budget: int = 1, pivot_rule: int = 0, weight_rule: int = 0,
+                set_rule: int = 0, pivot_key: Optional[torch.Tensor] = None) -> KvmParams:
+    """`pivot_key` ([batch, n_kv_heads, seq] fp32 CUDA tensor) must stay alive while the parameters are in use."""
     if isinstance(dtype, torch.dtype):
         dtype = {torch.bfloat16: KVM_BF16, torch.float32: KVM_F32}[dtype]
+    key_ptr = None
+    if pivot_key is not None:
+        assert pivot_key.is_cuda and pivot_key.dtype == torch.float32 and pivot_key.is_contiguous()
+        assert tuple(pivot_key.shape) == (batch, n_kv_heads, seq)
+        key_ptr = pivot_key.data_ptr()
     return KvmParams(batch, n_q_heads, n_kv_heads, seq, head_dim, int(dtype), budget, recent_ratio, heavy_ratio,
-                     sim_threshold, sigma, softmax_scale, causal, scale_v_by_set_size, enforce_budget)
+                     sim_threshold, sigma, softmax_scale, causal, scale_v_by_set_size, enforce_budget,
+                     pivot_rule, weight_rule, set_rule, key_ptr)
 
 
 def _ptr(t: Optional[torch.Tensor]) -> ctypes.c_void_p:

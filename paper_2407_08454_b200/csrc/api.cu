@@ -19,7 +19,6 @@ int derive(const kvm_params* p, Dims& d) {
     if (p->seq > KVM_MAX_SEQ) return KVM_E_SHAPE;
     if ((long long)p->batch * p->n_q_heads > 65535) return KVM_E_SHAPE;
     if (!(p->budget > 0.f && p->budget <= 1.f)) return KVM_E_PARAM;
-    if (!(p->sigma > 0.f) || !isfinite(p->sigma)) return KVM_E_PARAM;
     if (!isfinite(p->sim_threshold)) return KVM_E_PARAM;
     if (!isfinite(p->softmax_scale)) return KVM_E_PARAM;
     if (p->causal != 1) return KVM_E_UNSUPPORTED;
@@ -34,8 +33,23 @@ int derive(const kvm_params* p, Dims& d) {
     d.n_h = (int)floor((double)heavy * (double)d.S);
     d.enforce = p->enforce_budget ? 1 : 0;
     d.cap = d.enforce ? C : d.S;
-    // the forced cuts alone (first token, recent window, each heavy hitter and its right neighbour) must fit
-    if (d.enforce && (long long)d.cap < 1LL + d.n_r + 2LL * d.n_h) return KVM_E_PARAM;
+    if (p->pivot_rule < KVM_PIVOT_MAX_SCORE || p->pivot_rule > KVM_PIVOT_KEY) return KVM_E_PARAM;
+    if (p->weight_rule < KVM_WEIGHT_GAUSSIAN || p->weight_rule > KVM_WEIGHT_PIVOT_ONLY) return KVM_E_PARAM;
+    if (p->set_rule < KVM_SETS_ADJACENT || p->set_rule > KVM_SETS_CONSERVED_ONLY) return KVM_E_PARAM;
+    d.pivot_rule = p->pivot_rule; d.weight_rule = p->weight_rule; d.set_rule = p->set_rule;
+    d.pivot_key = p->pivot_key;
+    if (p->set_rule == KVM_SETS_ADJACENT && p->weight_rule == KVM_WEIGHT_GAUSSIAN &&
+        (!(p->sigma > 0.f) || !isfinite(p->sigma)))
+        return KVM_E_PARAM;
+    if (d.set_rule == KVM_SETS_CONSERVED_ONLY) {
+        d.pivot_rule = KVM_PIVOT_MAX_SCORE; d.weight_rule = KVM_WEIGHT_PIVOT_ONLY; d.pivot_key = nullptr;
+        if ((long long)d.cap < (long long)d.n_r + d.n_h) return KVM_E_PARAM;   // the kept tokens must fit
+    } else {
+        if (d.pivot_rule == KVM_PIVOT_KEY && !d.pivot_key) return KVM_E_NULL;
+        if (d.pivot_rule == KVM_PIVOT_KEY && ((uintptr_t)d.pivot_key & 15u)) return KVM_E_ALIGN;
+        // the forced cuts alone (first token, recent window, each heavy hitter and its right neighbour) must fit
+        if (d.enforce && (long long)d.cap < 1LL + d.n_r + 2LL * d.n_h) return KVM_E_PARAM;
+    }
     if (d.cap < 1) return KVM_E_PARAM;
     d.scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)d.D);
     d.eps = p->sim_threshold;
@@ -162,7 +176,8 @@ int kvm_segment(const kvm_params* p, const void* K, const float* scores, int32_t
     if ((rc = check_ws(d, ws, ws_bytes, w)) != KVM_OK) return rc;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     float* sim = sim_out ? sim_out : w.sim;
-    if (launch_similarity(d, K, sim, st) != cudaSuccess) return KVM_E_CUDA;
+    if (d.set_rule == KVM_SETS_ADJACENT || sim_out)
+        if (launch_similarity(d, K, sim, st) != cudaSuccess) return KVM_E_CUDA;
     if (launch_segment(d, scores, sim, set_id, set_start, pivot, out_len, stats, st) != cudaSuccess)
         return KVM_E_CUDA;
     return KVM_OK;
@@ -179,6 +194,10 @@ int kvm_merge_compact(const kvm_params* p, const void* K, const void* V, const i
     Workspace w;
     if ((rc = check_ws(d, ws, ws_bytes, w)) != KVM_OK) return rc;
     cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (d.weight_rule == KVM_WEIGHT_PIVOT_ONLY)
+        return launch_gather(d, K, V, set_start, pivot, out_len, K_out, V_out, out_size, st) == cudaSuccess
+                   ? KVM_OK
+                   : KVM_E_CUDA;
     if (launch_token_sets(d, set_start, out_len, w.set_id, st) != cudaSuccess) return KVM_E_CUDA;
     return launch_merge(d, K, V, set_start, pivot, w.set_id, K_out, V_out, out_size, w.merge_part, st) == cudaSuccess
                ? KVM_OK
@@ -200,9 +219,14 @@ int kvm_compress(const kvm_params* p, const void* Q, const void* K, const void* 
     cudaStream_t st = (cudaStream_t)cuda_stream;
     float* scores = scores_out ? scores_out : w.scores;
     if (run_score(d, Q, K, nullptr, scores, w, stats, st) != cudaSuccess) return KVM_E_CUDA;
-    if (launch_similarity(d, K, w.sim, st) != cudaSuccess) return KVM_E_CUDA;
+    if (d.set_rule == KVM_SETS_ADJACENT)
+        if (launch_similarity(d, K, w.sim, st) != cudaSuccess) return KVM_E_CUDA;
     if (launch_segment(d, scores, w.sim, w.set_id, w.set_start, out_pos, out_len, stats, st) != cudaSuccess)
         return KVM_E_CUDA;
+    if (d.weight_rule == KVM_WEIGHT_PIVOT_ONLY)
+        return launch_gather(d, K, V, w.set_start, out_pos, out_len, K_out, V_out, nullptr, st) == cudaSuccess
+                   ? KVM_OK
+                   : KVM_E_CUDA;
     if (launch_merge(d, K, V, w.set_start, out_pos, w.set_id, K_out, V_out, nullptr, w.merge_part, st) != cudaSuccess)
         return KVM_E_CUDA;
     return KVM_OK;

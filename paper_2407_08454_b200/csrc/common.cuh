@@ -15,6 +15,8 @@ struct Dims {
     int dtype;  // kvm_dtype
     float scale, eps, sigma;
     int scale_v, enforce;
+    int pivot_rule, weight_rule, set_rule;   // kvm_pivot_rule, kvm_weight_rule, kvm_set_rule
+    const float* pivot_key;                  // [U,S] when pivot_rule == KVM_PIVOT_KEY
 };
 
 // 16-byte vector <-> fp32 lanes.  Vec<T>::N elements of T per 16 bytes.
@@ -64,5 +66,9 @@ cudaError_t launch_token_sets(const Dims& d, const int32_t* set_start, const int
 cudaError_t launch_merge(const Dims& d, const void* K, const void* V, const int32_t* set_start,
                          const int32_t* pivot, const int32_t* set_id, void* K_out, void* V_out, int32_t* out_size,
                          float* scratch, cudaStream_t st);
+// Rows that are one input state each (pivot-only weights, eviction): a gather.
+cudaError_t launch_gather(const Dims& d, const void* K, const void* V, const int32_t* set_start,
+                          const int32_t* pivot, const int32_t* out_len, void* K_out, void* V_out, int32_t* out_size,
+                          cudaStream_t st);
 
 }  // namespace kvm

@@ -20,6 +20,8 @@
 // second kernel adds a crossing set's slots in tile order and stores the row.
 // Nothing uses atomics: every sum has a fixed order, results are reproducible.
 // Sets of one token are copied bit for bit.
+// Variants: average-weighted merging (Section 4.2) is the same kernel with every
+// g_j = 1; pivot-only weights and eviction write single input rows (gather_rows_kernel).
 #include "common.cuh"
 
 namespace kvm {
@@ -81,7 +83,8 @@ __global__ void __launch_bounds__(MERGE_NT) merge_tile_kernel(const T* __restric
                                                               const int32_t* __restrict__ set_id,
                                                               T* __restrict__ K_out, T* __restrict__ V_out,
                                                               int32_t* __restrict__ out_size, Slots<D> slots, int S,
-                                                              int cap, float neg_inv_2s2_log2e, int scale_v) {
+                                                              int cap, float neg_inv_2s2_log2e, int scale_v,
+                                                              int average) {
     using Gm = MergeGeom<T, D>;
     constexpr int N = Gm::N, LPR = Gm::LPR, NWORK = Gm::NWORK, NCH = Gm::NCH;
     constexpr int CHL = TOK / NCH;                    // tokens per chunk
@@ -150,7 +153,7 @@ __global__ void __launch_bounds__(MERGE_NT) merge_tile_kernel(const T* __restric
         for (int e = 0; e < N; ++e) { const float a = kp[e] - kj[e]; d2 = fmaf(a, a, d2); }
 #pragma unroll
         for (int off = 1; off < LPR; off <<= 1) d2 += __shfl_xor_sync(gmask, d2, off);
-        if (lane == 0) s_g[j] = exp2f(d2 * neg_inv_2s2_log2e);
+        if (lane == 0) s_g[j] = average ? 1.f : exp2f(d2 * neg_inv_2s2_log2e);
     }
     __syncthreads();
 
@@ -299,6 +302,48 @@ __global__ void __launch_bounds__(2 * D) merge_fixup_kernel(const int32_t* __res
     if (out_size && threadIdx.x == 0) out_size[(size_t)u * cap + sid] = n;
 }
 
+// Output rows that are a single input state: row s = K[pivot[s]], V[pivot[s]] (V times the set size when
+// asked and the sets are real ones).  One lane group per (row, tensor), 16-byte copies.
+template <typename T, int D>
+__global__ void __launch_bounds__(256) gather_rows_kernel(const T* __restrict__ K, const T* __restrict__ V,
+                                                          const int32_t* __restrict__ set_start,
+                                                          const int32_t* __restrict__ pivot,
+                                                          const int32_t* __restrict__ out_len, T* __restrict__ K_out,
+                                                          T* __restrict__ V_out, int32_t* __restrict__ out_size,
+                                                          int S, int cap, int scale_v, int singletons) {
+    constexpr int N = Vec<T>::N, LPR = D / N, ROWS = 256 / LPR / 2;
+    const long long u = blockIdx.y;
+    const int g = threadIdx.x / LPR, lane = threadIdx.x % LPR;
+    const int s = blockIdx.x * ROWS + (g >> 1), which = g & 1;
+    if (s >= min(out_len[u], cap)) return;
+    const int p = __ldg(pivot + (size_t)u * cap + s);
+    const int32_t* st = set_start + (size_t)u * (cap + 1);
+    const int n = singletons ? 1 : __ldg(st + s + 1) - __ldg(st + s);
+    const T* src = (which ? V : K) + ((size_t)u * S + p) * D + lane * N;
+    T* dst = (which ? V_out : K_out) + ((size_t)u * cap + s) * D + lane * N;
+    uint4 r = ldg16(src);
+    if (which && scale_v && n > 1) {
+        float x[N];
+        Vec<T>::unpack(r, x);
+#pragma unroll
+        for (int e = 0; e < N; ++e) x[e] *= (float)n;
+        r = Vec<T>::pack(x);
+    }
+    *reinterpret_cast<uint4*>(dst) = r;
+    if (out_size && which == 0 && lane == 0) out_size[(size_t)u * cap + s] = n;
+}
+
+template <typename T, int D>
+cudaError_t launch_gather_t(const Dims& d, const void* K, const void* V, const int32_t* set_start,
+                            const int32_t* pivot, const int32_t* out_len, void* K_out, void* V_out,
+                            int32_t* out_size, cudaStream_t st) {
+    constexpr int ROWS = 256 / (D / Vec<T>::N) / 2;
+    gather_rows_kernel<T, D><<<dim3((d.cap + ROWS - 1) / ROWS, d.U), 256, 0, st>>>(
+        (const T*)K, (const T*)V, set_start, pivot, out_len, (T*)K_out, (T*)V_out, out_size, d.S, d.cap, d.scale_v,
+        d.set_rule == KVM_SETS_CONSERVED_ONLY ? 1 : 0);
+    return cudaGetLastError();
+}
+
 template <typename T, int D, int TOK>
 cudaError_t launch_t(const Dims& d, const void* K, const void* V, const int32_t* set_start, const int32_t* pivot,
                      const int32_t* set_id, void* K_out, void* V_out, int32_t* out_size, float* scratch,
@@ -314,7 +359,7 @@ cudaError_t launch_t(const Dims& d, const void* K, const void* V, const int32_t*
     const float c = -LOG2E / (2.f * d.sigma * d.sigma);
     merge_tile_kernel<T, D, TOK><<<dim3(Tn, d.U), MERGE_NT, smem, st>>>(
         (const T*)K, (const T*)V, set_start, pivot, set_id, (T*)K_out, (T*)V_out, out_size, slots, d.S, d.cap, c,
-        d.scale_v);
+        d.scale_v, d.weight_rule == KVM_WEIGHT_AVERAGE ? 1 : 0);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     if (Tn > 1) {
         merge_fixup_kernel<T, D, TOK><<<dim3(Tn - 1, d.U), 2 * D, 0, st>>>(set_start, set_id, (T*)K_out, (T*)V_out,
@@ -342,6 +387,18 @@ cudaError_t launch_token_sets(const Dims& d, const int32_t* set_start, const int
                               cudaStream_t st) {
     token_set_kernel<<<dim3((d.S + 255) / 256, d.U), 256, 0, st>>>(set_start, out_len, set_id, d.S, d.cap);
     return cudaGetLastError();
+}
+
+cudaError_t launch_gather(const Dims& d, const void* K, const void* V, const int32_t* set_start,
+                          const int32_t* pivot, const int32_t* out_len, void* K_out, void* V_out, int32_t* out_size,
+                          cudaStream_t st) {
+    if (d.dtype == KVM_BF16) {
+        return d.D == 128
+                   ? launch_gather_t<__nv_bfloat16, 128>(d, K, V, set_start, pivot, out_len, K_out, V_out, out_size, st)
+                   : launch_gather_t<__nv_bfloat16, 64>(d, K, V, set_start, pivot, out_len, K_out, V_out, out_size, st);
+    }
+    return d.D == 128 ? launch_gather_t<float, 128>(d, K, V, set_start, pivot, out_len, K_out, V_out, out_size, st)
+                      : launch_gather_t<float, 64>(d, K, V, set_start, pivot, out_len, K_out, V_out, out_size, st);
 }
 
 cudaError_t launch_merge(const Dims& d, const void* K, const void* V, const int32_t* set_start,

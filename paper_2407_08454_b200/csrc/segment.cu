@@ -8,7 +8,10 @@
 //   3. budget rule: radix-select the soft cuts with the smallest similarity when
 //      the sets would exceed the capacity;
 //   4. inclusive scan of the flags -> set ids, set starts, set count;
-//   5. segmented arg-max of the scores -> one pivot per set.
+//   5. segmented arg-max of the scores -> one pivot per set (or of the token
+//      index / a caller-supplied key, for the variants of Sections 4.2 and 5.3).
+// In eviction mode (Section 2.2) steps 2-5 are replaced by a compaction of the
+// conserved tokens.
 // Every tie is broken toward the lower token index, and every reduction has a
 // fixed order, so the integer outputs are reproducible bit for bit.
 #include <limits.h>
@@ -127,7 +130,9 @@ __global__ void __launch_bounds__(NT) segment_unit_kernel(const float* __restric
                                                           const float* __restrict__ sim, int32_t* __restrict__ set_id,
                                                           int32_t* __restrict__ set_start, int32_t* __restrict__ pivot,
                                                           int32_t* __restrict__ out_len, kvm_stats* stats, int S,
-                                                          int cap, int n_r, int n_h, float eps, int enforce) {
+                                                          int cap, int n_r, int n_h, float eps, int enforce,
+                                                          int pivot_rule, const float* __restrict__ pivot_key,
+                                                          int set_rule) {
     extern __shared__ uint8_t flags[];  // [S]
     __shared__ Shared sh;
     const int u = blockIdx.x;
@@ -162,6 +167,38 @@ __global__ void __launch_bounds__(NT) segment_unit_kernel(const float* __restric
         }
     }
     __syncthreads();
+
+    int32_t* st = set_start + (size_t)u * (cap + 1);
+    int32_t* pv = pivot + (size_t)u * cap;
+
+    // ---- eviction (Section 2.2): the conserved tokens are the output, one state each
+    if (set_rule == KVM_SETS_CONSERVED_ONLY) {
+        int nk = 0;
+        for (int j = lo; j < hi; ++j) nk += (flags[j] & F_KEEP) ? 1 : 0;
+        int n_keep;
+        int id = block_exscan(nk, n_keep, sh);
+        for (int j = lo; j < hi; ++j) {
+            const bool k = (flags[j] & F_KEEP) != 0;
+            if (k && id < cap) { st[id] = j; pv[id] = j; }
+            if (set_id) set_id[(size_t)u * S + j] = k ? id : -1;
+            id += k;
+        }
+        if (threadIdx.x == 0) {
+            if (n_keep <= cap) st[n_keep] = S;
+            out_len[u] = n_keep;
+            if (stats) {
+                atomicMax(&stats->max_out_len, n_keep);
+                int old = stats->min_out_len;      // 0 means "unset"
+                while (old == 0 || n_keep < old) {
+                    const int prev = atomicCAS(&stats->min_out_len, old, n_keep);
+                    if (prev == old) break;
+                    old = prev;
+                }
+                atomicAdd((unsigned long long*)&stats->sum_out_len, (unsigned long long)n_keep);
+            }
+        }
+        return;
+    }
 
     // ---- 2. boundary flags
     int n_hard = 0, n_soft = 0, n_near = 0;
@@ -213,8 +250,6 @@ __global__ void __launch_bounds__(NT) segment_unit_kernel(const float* __restric
     for (int j = lo; j < hi; ++j) ncut += (flags[j] & F_CUT) ? 1 : 0;
     int n_sets;
     const int before = block_exscan(ncut, n_sets, sh);
-    int32_t* st = set_start + (size_t)u * (cap + 1);
-    int32_t* pv = pivot + (size_t)u * cap;
     {
         int id = before - 1;
         for (int j = lo; j < hi; ++j) {
@@ -242,7 +277,12 @@ __global__ void __launch_bounds__(NT) segment_unit_kernel(const float* __restric
         }
     }
 
-    // ---- 5. segmented arg-max: pivot of each set (ties: lowest index)
+    // ---- 5. segmented arg-max: pivot of each set (ties: lowest index).  The key is the score (Eq. 6),
+    // the token index (last-index pivot of the average-weighted baseline) or the caller's key array.
+    const float* pk = pivot_key ? pivot_key + (size_t)u * S : a;
+    auto key_of = [&](int j) -> float {
+        return pivot_rule == KVM_PIVOT_LAST ? (float)j : (pivot_rule == KVM_PIVOT_KEY ? pk[j] : a[j]);
+    };
     // Per thread: `head` = best of the tokens before the first cut in its range
     // (they belong to a set that started earlier), `run` = best since its last cut.
     Best head = {-INFINITY, INT_MAX}, run = {-INFINITY, INT_MAX};
@@ -257,7 +297,7 @@ __global__ void __launch_bounds__(NT) segment_unit_kernel(const float* __restric
             ++id;
             run = {-INFINITY, INT_MAX};
         }
-        run = better(run, Best{a[j], j});
+        run = better(run, Best{key_of(j), j});
     }
     if (!seen_cut) head = run;
     // Exclusive segmented scan over threads of (value = tail or whole range, flag = seen_cut).
@@ -320,7 +360,9 @@ cudaError_t launch_segment(const Dims& d, const float* scores, const float* sim,
         if (e != cudaSuccess) return e;
     }
     segment_unit_kernel<<<d.U, NT, (size_t)d.S, st>>>(scores, sim, set_id, set_start, pivot, out_len, stats, d.S,
-                                                     d.cap, d.n_r, d.n_h, d.eps, d.enforce);
+                                                     d.cap, d.n_r, d.n_h, d.eps, d.enforce, d.pivot_rule,
+                                                     d.pivot_rule == KVM_PIVOT_KEY ? d.pivot_key : nullptr,
+                                                     d.set_rule);
     return cudaGetLastError();
 }
 

@@ -52,6 +52,10 @@ class Case:
     scale: Optional[float] = None
     scale_v: bool = True
     enforce: bool = True
+    pivot_rule: int = 0
+    weight_rule: int = 0
+    set_rule: int = 0
+    pivot_key: Optional[torch.Tensor] = None      # [B,Hkv,S] fp32 (CPU) when pivot_rule is "key"
 
     def __post_init__(self):
         r, h = preset(self.budget)
@@ -62,10 +66,14 @@ class Case:
 
     def params(self) -> kvm.KvmParams:
         B, Hq, S, D = self.Q.shape
+        if self.pivot_key is not None and getattr(self, "_key_dev", None) is None:
+            self._key_dev = self.pivot_key.float().contiguous().cuda()      # kept alive with the case
         return kvm.make_params(B, Hq, self.K.shape[1], S, D, self.Q.dtype, budget=self.budget,
                                recent_ratio=self.recent, heavy_ratio=self.heavy, sim_threshold=self.eps,
                                sigma=self.sigma, softmax_scale=self.scale or 0.0,
-                               scale_v_by_set_size=int(self.scale_v), enforce_budget=int(self.enforce))
+                               scale_v_by_set_size=int(self.scale_v), enforce_budget=int(self.enforce),
+                               pivot_rule=self.pivot_rule, weight_rule=self.weight_rule, set_rule=self.set_rule,
+                               pivot_key=getattr(self, "_key_dev", None))
 
     def oracle_scale(self) -> float:
         D = self.Q.shape[-1]
@@ -140,11 +148,15 @@ def kv_error(gpu: np.ndarray, ref: np.ndarray) -> float:
     return float(np.max(np.abs(gpu.astype(np.float64) - ref) / den))
 
 
-def _chain(case: Case, scores: np.ndarray, sim: np.ndarray, cap: int, n_r: int, n_h: int):
+def _chain(case: Case, scores: np.ndarray, sim: np.ndarray, cap: int, n_r: int, n_h: int,
+           key: Optional[np.ndarray] = None):
     keep = kvmo.keep(scores, n_r, n_h)
     b, fired = kvmo.boundaries(sim, keep, cap, f32(case.eps), case.enforce)
     set_id, set_start, out_len = kvmo.sets(b, cap)
-    pivot = kvmo.pivots(scores, set_start, out_len)
+    if case.pivot_rule == kvm.KVM_PIVOT_LAST:
+        pivot = kvmo.pivots_last(set_start, out_len)
+    else:
+        pivot = kvmo.pivots(key if case.pivot_rule == kvm.KVM_PIVOT_KEY else scores, set_start, out_len)
     return dict(keep=keep, b=b, fired=fired, set_id=set_id, set_start=set_start, out_len=out_len, pivot=pivot)
 
 
@@ -169,7 +181,7 @@ def _near_tie_unit(case: Case, a: np.ndarray, c: np.ndarray, ch: Dict[str, np.nd
     if np.any(np.abs(c[~hard] - f32(case.eps)) < NEAR_SIM):
         return True
     st, n = ch["set_start"][u], ch["out_len"][u]
-    for s in range(n):
+    for s in range(n if case.pivot_rule == kvm.KVM_PIVOT_MAX_SCORE else 0):
         lo, hi = st[s], st[s + 1]
         if hi - lo >= 2:
             top = np.sort(a[lo:hi])[-2:]
@@ -222,8 +234,11 @@ def check_case(case: Case, g: Optional[GpuOut] = None, units: Optional[list] = N
     assert rep.sim_err <= SIM_ATOL, f"similarity off by {rep.sim_err}"
 
     # integers: forced chain (checker fed the library's own fp32 scores and similarities)
-    forced = _chain(case, g_scores.astype(np.float64), g_sim.astype(np.float64), cap, n_r, n_h)
-    pure = _chain(case, ref_scores, ref_sim, cap, n_r, n_h)
+    key = None
+    if case.pivot_key is not None:
+        key = case.pivot_key.float().numpy().reshape(U, S)[sel].astype(np.float64)
+    forced = _chain(case, g_scores.astype(np.float64), g_sim.astype(np.float64), cap, n_r, n_h, key)
+    pure = _chain(case, ref_scores, ref_sim, cap, n_r, n_h, key)
     g_len = unit_view(g.out_len, ())
     g_st, g_pv, g_id = unit_view(g.set_start, (cap + 1,)), unit_view(g.pivot, (cap,)), unit_view(g.set_id, (S,))
     g_sz = unit_view(g.out_size, (cap,))
@@ -253,7 +268,8 @@ def check_case(case: Case, g: Optional[GpuOut] = None, units: Optional[list] = N
         assert np.array_equal(c_K[i, :n], g_K[i, :n]) and np.array_equal(c_V[i, :n], g_V[i, :n])
 
     # merged states: checker with the library's integer decisions forced in
-    rK, rV = kvmo.merge(Ks[:, 0], Vs[:, 0], g_st, np.where(g_pv < 0, 0, g_pv), g_len, f32(case.sigma), case.scale_v)
+    rK, rV = kvmo.merge(Ks[:, 0], Vs[:, 0], g_st, np.where(g_pv < 0, 0, g_pv), g_len, f32(case.sigma), case.scale_v,
+                        weight_rule=case.weight_rule)
     K32, V32 = Ks[:, 0].float().numpy(), Vs[:, 0].float().numpy()
     for i in range(len(sel)):
         n = g_len[i]
@@ -263,6 +279,10 @@ def check_case(case: Case, g: Optional[GpuOut] = None, units: Optional[list] = N
         single = np.nonzero(np.diff(g_st[i, : n + 1]) == 1)[0]
         assert np.array_equal(g_K[i, single], K32[i, g_st[i, single]]), "singleton rows must be bit-identical"
         assert np.array_equal(g_V[i, single], V32[i, g_st[i, single]])
+        if case.weight_rule == kvm.KVM_WEIGHT_PIVOT_ONLY:      # the pivot's own rows, whatever the set size
+            assert np.array_equal(g_K[i, :n], K32[i, g_pv[i, :n]])
+            if not case.scale_v:
+                assert np.array_equal(g_V[i, :n], V32[i, g_pv[i, :n]])
     assert rep.k_err <= KV_TOL, f"K_out error {rep.k_err}"
     assert rep.v_err <= KV_TOL, f"V_out error {rep.v_err}"
     return rep
@@ -293,3 +313,55 @@ def check_invariants_all_units(case: Case, g: GpuOut) -> None:
         assert ((pos[u, :n] >= st[u, :n]) & (pos[u, :n] < st[u, 1: n + 1])).all(), "pivot outside its set"
         single = np.nonzero(np.diff(st[u, : n + 1]) == 1)[0]
         assert np.array_equal(cK[u, single], K32[u, st[u, single]])
+
+
+def check_evict_case(case: Case, g: Optional[GpuOut] = None) -> Report:
+    """Parity of the eviction mode (only the conserved tokens stay).  The floating-point part is the
+    scores; given them every output is an integer or a copied row, so everything else is bit-exact
+    against the checker fed the library's own scores."""
+    assert case.set_rule == kvm.KVM_SETS_CONSERVED_ONLY
+    if g is None:
+        g = run_gpu(case)
+    B, Hq, S, D = case.Q.shape
+    Hkv = case.K.shape[1]
+    G, U = Hq // Hkv, B * Hkv
+    cap, n_r, n_h = kvm.kvm_sizes(case.params())
+    assert (cap, n_r, n_h) == _oracle_sizes(case, S)
+    rep = Report(units=U)
+    Qs = case.Q.reshape(U, G, S, D)
+    Ks, Vs = case.K.reshape(U, S, D), case.V.reshape(U, S, D)
+    ref_scores = kvmo.scores(Qs, Ks[:, None], scale=case.oracle_scale())[:, 0]
+    g_scores = g.scores.reshape(U, S)
+    rep.score_excess = score_excess(g_scores, ref_scores)
+    assert rep.score_excess <= 1.0
+    keep_forced = kvmo.keep(g_scores.astype(np.float64), n_r, n_h)
+    keep_pure = kvmo.keep(ref_scores, n_r, n_h)
+    r_len, r_pos, rK, rV = kvmo.evict(keep_forced, Ks, Vs, cap)
+    g_len, g_pv = g.out_len.reshape(U), g.pivot.reshape(U, cap)
+    g_st, g_id = g.set_start.reshape(U, cap + 1), g.set_id.reshape(U, S)
+    assert np.array_equal(g_len, r_len) and (g_len == min(S, n_r) + min(n_h, max(0, S - n_r))).all()
+    for name, step, comp in (("K", g.K_out, g.c_K_out), ("V", g.V_out, g.c_V_out)):
+        ref = rK if name == "K" else rV
+        step, comp = step.reshape(U, cap, D), comp.reshape(U, cap, D)
+        for u in range(U):
+            n = g_len[u]
+            assert np.array_equal(step[u, :n].astype(np.float64), ref[u, :n]), f"{name}_out rows, unit {u}"
+            assert np.array_equal(comp[u, :n], step[u, :n])
+            assert (step[u, n:] == 768.0).all() and (comp[u, n:] == 768.0).all()
+    for u in range(U):
+        n = g_len[u]
+        assert np.array_equal(g_pv[u, :n], r_pos[u, :n]) and (g_pv[u, n:] == -7).all()
+        assert np.array_equal(g_st[u, :n], r_pos[u, :n]) and g_st[u, n] == S
+        kf = keep_forced[u].astype(np.int64)
+        want_id = np.where(kf != 0, np.cumsum(kf) - 1, -1)
+        assert np.array_equal(g_id[u], want_id)
+        assert np.array_equal(g.out_size.reshape(U, cap)[u, :n], np.ones(n, np.int32))
+        assert np.array_equal(g.c_out_pos.reshape(U, cap)[u, :n], r_pos[u, :n])
+        if not np.array_equal(keep_forced[u], keep_pure[u]):
+            rep.units_differ_from_fp64_chain += 1
+            R = max(0, S - n_r)
+            srt = np.sort(ref_scores[u, :R])[::-1]
+            assert srt[n_h - 1] - srt[n_h] < NEAR_SCORE * srt[n_h - 1], f"unit {u}: kept set differs without a near-tie"
+            rep.units_near_tie += 1
+    assert np.array_equal(g.c_out_len.reshape(U), g_len)
+    return rep

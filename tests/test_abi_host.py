@@ -27,7 +27,8 @@ def test_every_declared_symbol_is_exported(lib):
         assert hasattr(lib, name), name
     assert declared == set(binding.EXPORTS) | (declared - set(binding.EXPORTS))
     assert set(binding.EXPORTS) <= declared
-    assert kvm.kvm_version() == 100
+    assert kvm.kvm_version() == 101
+    assert ctypes.sizeof(kvm.KvmParams) == 80 and kvm.KvmParams.pivot_key.offset == 72
 
 
 def test_sizes_and_presets(lib):
@@ -62,6 +63,28 @@ def test_bad_parameters_are_rejected_on_the_host(lib, kw, status):
     n = ctypes.c_size_t()
     assert lib.kvm_workspace_bytes(ctypes.byref(p), ctypes.byref(n)) == status
     assert kvm.status_string(status) != "unknown status"
+
+
+def test_variant_parameter_checks(lib):
+    p = kvm.make_params(1, 2, 2, 256, 64, kvm.KVM_F32, pivot_rule=kvm.KVM_PIVOT_KEY)     # key missing
+    with pytest.raises(kvm.KvmError) as e:
+        kvm.kvm_sizes(p)
+    assert e.value.status == -1
+    for bad in (dict(pivot_rule=3), dict(weight_rule=-1), dict(set_rule=2)):
+        with pytest.raises(kvm.KvmError) as e:
+            kvm.kvm_sizes(kvm.make_params(1, 2, 2, 256, 64, kvm.KVM_F32, **bad))
+        assert e.value.status == -4
+    # eviction: the kept tokens must fit the capacity
+    with pytest.raises(kvm.KvmError) as e:
+        kvm.kvm_sizes(kvm.make_params(1, 2, 2, 256, 64, kvm.KVM_F32, budget=0.5, recent_ratio=0.3, heavy_ratio=0.3,
+                                      set_rule=kvm.KVM_SETS_CONSERVED_ONLY))
+    assert e.value.status == -4
+    # ... while the same shares are fine when they fill it exactly, which Algorithm 1's forced cuts would not allow
+    assert kvm.kvm_sizes(kvm.make_params(1, 2, 2, 256, 64, kvm.KVM_F32, budget=0.5, recent_ratio=0.25,
+                                         heavy_ratio=0.25, set_rule=kvm.KVM_SETS_CONSERVED_ONLY))[0] == 128
+    # average weights ignore sigma
+    assert kvm.kvm_sizes(kvm.make_params(1, 2, 2, 256, 64, kvm.KVM_F32, sigma=0.0,
+                                         weight_rule=kvm.KVM_WEIGHT_AVERAGE))[0] == 128
 
 
 def test_null_alignment_and_workspace_errors(lib):
