@@ -196,6 +196,18 @@ int kvm_compress_host(const kvm_params* p, const void* Q, const void* K, const v
                       void* dev, size_t dev_bytes, void* cuda_stream);
 
 /*
+ * Layer-wise compression ratio of the set identification alone (Section 3.2, Figure 3(b)): per unit,
+ * (number of merging sets Algorithm 1 forms with nothing conserved and no budget) / S, for the
+ * threshold p->sim_threshold.  Lowering the threshold lowers the ratio; the paper proposes choosing a
+ * threshold per layer from this statistic, which callers do by giving each layer's kvm_compress call its
+ * own sim_threshold.
+ *   K [batch, n_kv_heads, S, D]; ratio [U] fp32 (device), written; sim_out NULL or [U, S] fp32.
+ * budget, recent_ratio, heavy_ratio, sigma and the rules of p are not used.
+ */
+int kvm_layer_ratio(const kvm_params* p, const void* K, float* ratio, float* sim_out,
+                    void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
  * kvm_score for callers that cannot allocate device memory.  (The paper has no
  * counterpart: this is a packaging variant of kvm_score, same arithmetic.)
  *

@@ -178,6 +178,24 @@ void kvmo_boundaries(int64_t U, int32_t S, int32_t C, double eps, int32_t enforc
     }
 }
 
+// Layer-wise compression ratio of Section 3.2 (Figure 3(b)): the number of
+// groups the set identification forms on its own -- walking the sequence and
+// grouping a state with its neighbour while their similarity exceeds eps, with
+// nothing conserved and no budget -- over the number of states.  ratio [U].
+void kvmo_layer_ratio(int64_t U, int32_t S, double eps, const double* sim, double* ratio) {
+    for (int64_t u = 0; u < U; ++u) {
+        int32_t groups = 0;
+        int32_t i = S - 1;                       // from the last token to the first
+        while (i >= 0) {
+            ++groups;
+            int32_t j = i - 1;
+            while (j >= 0 && sim[(size_t)u * S + j + 1] > eps) --j;   // sim_{j+1} pairs tokens j and j+1
+            i = j;
+        }
+        ratio[u] = (double)groups / (double)S;
+    }
+}
+
 // Definition 4.1's partition: consecutive, disjoint sets covering the sequence.
 // set_id_j = (number of flags at positions <= j) - 1; set s = [set_start[s], set_start[s+1]).
 // set_id [U,S]; set_start [U,cap+1]; out_len [U].  Entries past out_len are untouched.

@@ -102,6 +102,15 @@ def boundaries(sim: np.ndarray, keep_: np.ndarray, C: int, eps: float, enforce_b
     return b, fired
 
 
+def layer_ratio(sim: np.ndarray, eps: float) -> np.ndarray:
+    sim = np.ascontiguousarray(sim, dtype=np.float64)
+    S = sim.shape[-1]
+    U = sim.size // S
+    out = np.empty(sim.shape[:-1], dtype=np.float64)
+    lib().kvmo_layer_ratio(ctypes.c_int64(U), ctypes.c_int32(S), ctypes.c_double(eps), _p(sim), _p(out))
+    return out
+
+
 def sets(b: np.ndarray, cap: int):
     b = np.ascontiguousarray(b, dtype=np.uint8)
     S = b.shape[-1]

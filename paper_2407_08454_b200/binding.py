@@ -24,7 +24,8 @@ KVM_WEIGHT_GAUSSIAN, KVM_WEIGHT_AVERAGE, KVM_WEIGHT_PIVOT_ONLY = 0, 1, 2
 KVM_SETS_ADJACENT, KVM_SETS_CONSERVED_ONLY = 0, 1
 EXPORTS = (
     "kvm_sizes", "kvm_workspace_bytes", "kvm_score", "kvm_segment", "kvm_merge_compact", "kvm_compress",
-    "kvm_host_staging_bytes", "kvm_compress_host", "kvm_score_static", "kvm_status_string", "kvm_version",
+    "kvm_host_staging_bytes", "kvm_compress_host", "kvm_score_static", "kvm_layer_ratio", "kvm_status_string",
+    "kvm_version",
 )
 KVM_STATIC_SCORE_ROWS = 1 << 20
 
@@ -158,6 +159,11 @@ def kvm_segment(p: KvmParams, K, scores, set_id, set_start, pivot, out_len, sim_
                              ctypes.c_size_t(ws.numel() * ws.element_size()), _stream(stream)), "kvm_segment")
 
 
+def kvm_layer_ratio(p: KvmParams, K, ratio, sim_out, ws, stream=None) -> None:
+    _check(lib().kvm_layer_ratio(ctypes.byref(p), _ptr(K), _ptr(ratio), _ptr(sim_out), _ptr(ws),
+                                 ctypes.c_size_t(ws.numel() * ws.element_size()), _stream(stream)), "kvm_layer_ratio")
+
+
 def kvm_merge_compact(p: KvmParams, K, V, set_start, pivot, out_len, K_out, V_out, out_size, ws, stream=None) -> None:
     _check(lib().kvm_merge_compact(ctypes.byref(p), _ptr(K), _ptr(V), _ptr(set_start), _ptr(pivot), _ptr(out_len),
                                    _ptr(K_out), _ptr(V_out), _ptr(out_size), _ptr(ws),
@@ -219,3 +225,22 @@ class Compressor:
         kvm_compress(self.p, Q, K, V, self.K_out, self.V_out, self.out_len, self.out_pos, self.scores, stats,
                      self.ws, stream)
         return Compressed(self.K_out, self.V_out, self.out_len, self.out_pos, self.scores, self.cap)
+
+
+def compress_layers(p: KvmParams, layers, sim_thresholds=None, device="cuda", stream=None):
+    """Compress a stack of layers, each an (Q, K, V) triple of CUDA tensors of the shape `p` describes, with one
+    similarity threshold per layer (Section 3.2: thresholds chosen layer by layer).  Returns, per layer, a
+    `Compressed` holding copies of the outputs, and the layer's compression ratio mean(out_len) / S."""
+    n = len(layers)
+    if sim_thresholds is None:
+        sim_thresholds = [p.sim_threshold] * n
+    assert len(sim_thresholds) == n
+    out, ratios = [], []
+    for (Q, K, V), eps in zip(layers, sim_thresholds):
+        pl = KvmParams.from_buffer_copy(bytes(p))
+        pl.sim_threshold = float(eps)
+        c = Compressor(pl, device=device)
+        r = c(Q, K, V, stream=stream)
+        out.append(r)
+        ratios.append(r.out_len.float().mean() / p.seq)
+    return out, [float(x) for x in ratios]

@@ -183,6 +183,21 @@ int kvm_segment(const kvm_params* p, const void* K, const float* scores, int32_t
     return KVM_OK;
 }
 
+int kvm_layer_ratio(const kvm_params* p, const void* K, float* ratio, float* sim_out, void* ws, size_t ws_bytes,
+                    void* cuda_stream) {
+    Dims d;
+    int rc = derive(p, d);
+    if (rc != KVM_OK) return rc;
+    if (!K || !ratio) return KVM_E_NULL;
+    if (misaligned(K)) return KVM_E_ALIGN;
+    Workspace w;
+    if ((rc = check_ws(d, ws, ws_bytes, w)) != KVM_OK) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    float* sim = sim_out ? sim_out : w.sim;
+    if (launch_similarity(d, K, sim, st) != cudaSuccess) return KVM_E_CUDA;
+    return launch_set_ratio(d, sim, ratio, st) == cudaSuccess ? KVM_OK : KVM_E_CUDA;
+}
+
 int kvm_merge_compact(const kvm_params* p, const void* K, const void* V, const int32_t* set_start,
                       const int32_t* pivot, const int32_t* out_len, void* K_out, void* V_out, int32_t* out_size,
                       void* ws, size_t ws_bytes, void* cuda_stream) {

@@ -350,7 +350,31 @@ __global__ void __launch_bounds__(NT) segment_unit_kernel(const float* __restric
     }
 }
 
+// Sets formed by Algorithm 1 alone (nothing conserved, no budget) over the sequence length:
+// 1 + #{j >= 1 : not (sim_j > eps)}, divided by S.  One block per unit.
+__global__ void __launch_bounds__(256) set_ratio_kernel(const float* __restrict__ sim, float* __restrict__ ratio,
+                                                        int S, float eps) {
+    __shared__ int part[8];
+    const float* c = sim + (size_t)blockIdx.x * S;
+    int n = 0;
+    for (int j = 1 + threadIdx.x; j < S; j += 256) n += !(c[j] > eps);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) n += __shfl_xor_sync(0xffffffffu, n, off);
+    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = n;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int t = 1;
+        for (int w = 0; w < 8; ++w) t += part[w];
+        ratio[blockIdx.x] = (float)t / (float)S;
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_set_ratio(const Dims& d, const float* sim, float* ratio, cudaStream_t st) {
+    set_ratio_kernel<<<d.U, 256, 0, st>>>(sim, ratio, d.S, d.eps);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_segment(const Dims& d, const float* scores, const float* sim, int32_t* set_id,
                            int32_t* set_start, int32_t* pivot, int32_t* out_len, kvm_stats* stats, cudaStream_t st) {

@@ -65,3 +65,34 @@ def test_eviction_keeps_the_conserved_tokens(name, kw):
     case = _case(name, kw, set_rule=kvm.KVM_SETS_CONSERVED_ONLY, recent=recent, heavy=cfg.budget - recent)
     rep = check_evict_case(case)
     print(name, kw, rep)
+
+
+def test_layer_ratio_and_per_layer_thresholds():
+    # per-layer token correlation differs (as across a model's layers): the ratio statistic follows it, and a
+    # threshold per layer steers it (Section 3.2)
+    cfg = si.CONFIGS["C2"].scaled(seq=1024, n_q_heads=4, n_kv_heads=4, batch=1, layers=4)
+    from oracle import kvmo
+    p = kvm.make_params(1, 4, 4, 1024, 128, torch.bfloat16, budget=cfg.budget)
+    ws = torch.empty(kvm.kvm_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+    layers, ratios = [], []
+    for layer in range(4):
+        d = si.make_layer(cfg, layer)
+        K = d["K"].cuda()
+        layers.append((d["Q"].cuda(), K, d["V"].cuda()))
+        ratio = torch.full((4,), -1.0, device="cuda")
+        sim = torch.empty(1, 4, 1024, device="cuda")
+        kvm.kvm_layer_ratio(p, K, ratio, sim, ws)
+        ref_sim = kvmo.similarity(d["K"][0])
+        assert np.abs(sim[0].cpu().numpy() - ref_sim).max() <= 4e-6
+        want = kvmo.layer_ratio(sim[0].double().cpu().numpy(), float(np.float32(0.75)))     # same fp32 similarities
+        np.testing.assert_allclose(ratio.cpu().numpy(), want, rtol=1e-6)
+        ratios.append(float(ratio.mean()))
+        assert 1.0 / 1024 <= ratios[-1] <= 1.0
+    # per-layer thresholds through the whole path: a lower threshold never gives more rows
+    outs_hi, r_hi = kvm.compress_layers(p, layers, [0.9] * 4)
+    outs_lo, r_lo = kvm.compress_layers(p, layers, [0.6, 0.65, 0.7, 0.75])
+    assert all(lo <= hi for lo, hi in zip(r_lo, r_hi))
+    for (Q, K, V), o, eps in zip(layers, outs_lo, [0.6, 0.65, 0.7, 0.75]):
+        g = run_gpu(Case(Q.cpu(), K.cpu(), V.cpu(), budget=cfg.budget, eps=eps))
+        assert np.array_equal(o.out_len.cpu().numpy(), g.c_out_len)
+    print("layer ratios", ratios, "compressed", r_lo, r_hi)

@@ -142,3 +142,36 @@ def test_compress_variants_equal_their_steps():
         np.testing.assert_array_equal(r.pivot[0, u, :n], idx)
         np.testing.assert_array_equal(r.K_out[0, u, :n], K64[0, u, idx])
         assert (r.set_id[0, u, idx] == np.arange(n)).all() and (np.delete(r.set_id[0, u], idx) == -1).all()
+
+
+def test_layer_ratio_walk_equals_flag_count_and_limits():
+    # the backward walk of Section 3.2 and the forward boundary flags of Algorithm 1 count the same groups
+    rng = np.random.default_rng(14)
+    sim = rng.uniform(0.4, 1.0, (5, 300))
+    sim[:, 0] = 0
+    none = np.zeros((5, 300), np.uint8)
+    for eps in (0.5, 0.75, 0.9):
+        b, _ = kvmo.boundaries(sim, none, C=300, eps=eps, enforce_budget=False)
+        np.testing.assert_array_equal(kvmo.layer_ratio(sim, eps), b.sum(-1) / 300.0)
+    r = [kvmo.layer_ratio(sim, e).mean() for e in np.linspace(0.3, 1.0, 15)]
+    assert all(x <= y for x, y in zip(r, r[1:]))                         # lower threshold -> fewer groups
+    ident = np.repeat(_rand((1, 1, 8), 15), 40, axis=1)
+    assert kvmo.layer_ratio(kvmo.similarity(ident), 0.75)[0] == 1 / 40  # one group
+    assert kvmo.layer_ratio(kvmo.similarity(np.eye(8, dtype=np.float32)[None]), 0.75)[0] == 1.0
+    # brute force on a hand-made row: similar pairs (1,2), (2,3) and (5,6) -> groups {0},{1,2,3},{4},{5,6}
+    row = np.array([[0.0, 0.1, 0.9, 0.8, 0.2, 0.3, 0.99]])
+    assert kvmo.layer_ratio(row, 0.75)[0] == 4 / 7
+
+
+def test_layer_ratio_of_wide_ar1_keys_is_a_step_in_rho():
+    # for many channels the cosine of AR(1) neighbours concentrates at rho: all in one group below it, none above
+    rng = np.random.default_rng(16)
+    S, D, rho = 64, 8192, 0.9
+    x = np.empty((S, D))
+    x[0] = rng.standard_normal(D)
+    for t in range(1, S):
+        x[t] = rho * x[t - 1] + np.sqrt(1 - rho * rho) * rng.standard_normal(D)
+    sim = kvmo.similarity(x[None].astype(np.float32))
+    assert np.abs(sim[0, 1:] - rho).max() < 0.02
+    assert kvmo.layer_ratio(sim, rho - 0.05)[0] == 1 / S
+    assert kvmo.layer_ratio(sim, rho + 0.05)[0] == 1.0
