@@ -314,6 +314,54 @@ void kvmo_evict(int64_t U, int32_t S, int32_t D, int32_t cap, const uint8_t* kee
     }
 }
 
+// One decode step of Eq. 1 over a cache that may be compressed: for query head
+// h of batch entry b (KV head h / G), with the first len[u] of `rows` cache rows,
+//   A_t = softmax(scale * q_t K^T),   O_t = A_t V.
+// q [B,Hq,D]; K, V [B,Hkv,rows,D]; len [B*Hkv] (nullable: all rows); out [B,Hq,D].
+// No rows -> O_t = 0.
+void kvmo_attend(int32_t B, int32_t Hq, int32_t Hkv, int32_t rows, int32_t D, double scale,
+                 const float* q, const float* K, const float* V, const int32_t* len, double* out) {
+    const int32_t G = Hq / Hkv;
+    for (int32_t b = 0; b < B; ++b)
+        for (int32_t h = 0; h < Hq; ++h) {
+            const int64_t u = (int64_t)b * Hkv + h / G;
+            const int32_t n = len ? len[u] : rows;
+            const float* qt = q + ((size_t)b * Hq + h) * D;
+            const float* Ku = K + (size_t)u * rows * D;
+            const float* Vu = V + (size_t)u * rows * D;
+            double* o = out + ((size_t)b * Hq + h) * D;
+            for (int32_t t = 0; t < D; ++t) o[t] = 0.0;
+            if (n <= 0) continue;
+            std::vector<double> s(n);
+            double m = -INFINITY;
+            for (int32_t j = 0; j < n; ++j) {
+                double dot = 0.0;
+                for (int32_t t = 0; t < D; ++t) dot += (double)qt[t] * (double)Ku[(size_t)j * D + t];
+                s[j] = scale * dot;
+                m = std::max(m, s[j]);
+            }
+            double l = 0.0;
+            for (int32_t j = 0; j < n; ++j) { s[j] = std::exp(s[j] - m); l += s[j]; }
+            for (int32_t j = 0; j < n; ++j)
+                for (int32_t t = 0; t < D; ++t) o[t] += (s[j] / l) * (double)Vu[(size_t)j * D + t];
+        }
+}
+
+// Definition 2.1's criterion |O_t - O_t*|, read as the Euclidean norm per
+// attention head; ref = |O_t| for a relative figure.  O, O_star [n,D]; err, ref [n].
+void kvmo_perturbation(int64_t n, int32_t D, const double* O, const double* O_star, double* err, double* ref) {
+    for (int64_t i = 0; i < n; ++i) {
+        double e = 0.0, r = 0.0;
+        for (int32_t t = 0; t < D; ++t) {
+            const double d = O[(size_t)i * D + t] - O_star[(size_t)i * D + t];
+            e += d * d;
+            r += O[(size_t)i * D + t] * O[(size_t)i * D + t];
+        }
+        err[i] = std::sqrt(e);
+        ref[i] = std::sqrt(r);
+    }
+}
+
 // The whole path for one layer, steps in the paper's order.  All outputs are
 // caller-allocated; cap = C when enforce_budget, else S.
 // Variants (all 0 = the paper's method): pivot_rule 1 = last index of the set,

@@ -187,6 +187,34 @@ def merge(K, V, set_start, pivot, out_len, sigma: float, scale_v: bool = True, w
     return (Ko, Vo, w) if want_weights else (Ko, Vo)
 
 
+def attend(q, K, V, length=None, scale: Optional[float] = None) -> np.ndarray:
+    """One decode step (Eq. 1): q [B,Hq,D], K/V [B,Hkv,rows,D], length [B,Hkv] or None -> O [B,Hq,D] fp64."""
+    q, K, V = _f32(q), _f32(K), _f32(V)
+    B, Hq, D = q.shape
+    Hkv, rows = K.shape[1], K.shape[2]
+    if scale is None:
+        scale = 1.0 / math.sqrt(D)
+    if length is not None:
+        length = np.ascontiguousarray(length, dtype=np.int32)
+        assert length.size == B * Hkv
+    out = np.empty((B, Hq, D), dtype=np.float64)
+    lib().kvmo_attend(ctypes.c_int32(B), ctypes.c_int32(Hq), ctypes.c_int32(Hkv), ctypes.c_int32(rows),
+                      ctypes.c_int32(D), ctypes.c_double(scale), _p(q), _p(K), _p(V), _p(length), _p(out))
+    return out
+
+
+def perturbation(O: np.ndarray, O_star: np.ndarray):
+    """Definition 2.1's |O_t - O_t*| per head (Euclidean norm) and |O_t|."""
+    O = np.ascontiguousarray(O, dtype=np.float64)
+    O_star = np.ascontiguousarray(O_star, dtype=np.float64)
+    D = O.shape[-1]
+    n = O.size // D
+    err = np.empty(O.shape[:-1], dtype=np.float64)
+    ref = np.empty(O.shape[:-1], dtype=np.float64)
+    lib().kvmo_perturbation(ctypes.c_int64(n), ctypes.c_int32(D), _p(O), _p(O_star), _p(err), _p(ref))
+    return err, ref
+
+
 @dataclass
 class Compressed:
     scores: np.ndarray
