@@ -208,6 +208,28 @@ int kvm_layer_ratio(const kvm_params* p, const void* K, float* ratio, float* sim
                     void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * One decode step of attention (Eq. 1: O_t = softmax(q_t K^T * scale) V) over a cache whose units may hold
+ * different numbers of rows, e.g. the output of kvm_compress.  Query head h of batch entry b reads KV head h / G.
+ *   q    [batch, n_q_heads, D] in p->dtype
+ *   K, V [batch, n_kv_heads, rows, D] in p->dtype, 1 <= rows <= S
+ *   len  NULL (every unit holds `rows` rows) or device [U] i32: rows of each unit that are valid
+ *   out  [batch, n_q_heads, D] fp32, written; a unit with no rows gives zeros
+ * fp32 arithmetic.  Only the shape, dtype and softmax_scale of p are used.
+ */
+int kvm_attend(const kvm_params* p, const void* q, const void* K, const void* V, int32_t rows, const int32_t* len,
+               float* out, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * The criterion of Definition 2.1 for one decode step: attention outputs over the full cache (K, V
+ * [U, S, D]) and over the compressed one (K_c, V_c [U, cap, D] with len_c [U], as kvm_compress leaves
+ * them for the same p), and per (batch, query head) err = |O_t - O_t*|_2 and ref = |O_t|_2.
+ *   out_full, out_comp [batch, n_q_heads, D] fp32; err, ref [batch, n_q_heads] fp32; all written.
+ */
+int kvm_output_perturbation(const kvm_params* p, const void* q, const void* K, const void* V, const void* K_c,
+                            const void* V_c, const int32_t* len_c, float* out_full, float* out_comp, float* err,
+                            float* ref, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
  * kvm_score for callers that cannot allocate device memory.  (The paper has no
  * counterpart: this is a packaging variant of kvm_score, same arithmetic.)
  *

@@ -24,7 +24,8 @@ KVM_WEIGHT_GAUSSIAN, KVM_WEIGHT_AVERAGE, KVM_WEIGHT_PIVOT_ONLY = 0, 1, 2
 KVM_SETS_ADJACENT, KVM_SETS_CONSERVED_ONLY = 0, 1
 EXPORTS = (
     "kvm_sizes", "kvm_workspace_bytes", "kvm_score", "kvm_segment", "kvm_merge_compact", "kvm_compress",
-    "kvm_host_staging_bytes", "kvm_compress_host", "kvm_score_static", "kvm_layer_ratio", "kvm_status_string",
+    "kvm_host_staging_bytes", "kvm_compress_host", "kvm_score_static", "kvm_layer_ratio", "kvm_attend",
+    "kvm_output_perturbation", "kvm_status_string",
     "kvm_version",
 )
 KVM_STATIC_SCORE_ROWS = 1 << 20
@@ -162,6 +163,19 @@ def kvm_segment(p: KvmParams, K, scores, set_id, set_start, pivot, out_len, sim_
 def kvm_layer_ratio(p: KvmParams, K, ratio, sim_out, ws, stream=None) -> None:
     _check(lib().kvm_layer_ratio(ctypes.byref(p), _ptr(K), _ptr(ratio), _ptr(sim_out), _ptr(ws),
                                  ctypes.c_size_t(ws.numel() * ws.element_size()), _stream(stream)), "kvm_layer_ratio")
+
+
+def kvm_attend(p: KvmParams, q, K, V, rows: int, length, out, ws, stream=None) -> None:
+    _check(lib().kvm_attend(ctypes.byref(p), _ptr(q), _ptr(K), _ptr(V), ctypes.c_int32(rows), _ptr(length), _ptr(out),
+                            _ptr(ws), ctypes.c_size_t(ws.numel() * ws.element_size()), _stream(stream)), "kvm_attend")
+
+
+def kvm_output_perturbation(p: KvmParams, q, K, V, K_c, V_c, len_c, out_full, out_comp, err, ref, ws,
+                            stream=None) -> None:
+    _check(lib().kvm_output_perturbation(ctypes.byref(p), _ptr(q), _ptr(K), _ptr(V), _ptr(K_c), _ptr(V_c),
+                                         _ptr(len_c), _ptr(out_full), _ptr(out_comp), _ptr(err), _ptr(ref), _ptr(ws),
+                                         ctypes.c_size_t(ws.numel() * ws.element_size()), _stream(stream)),
+           "kvm_output_perturbation")
 
 
 def kvm_merge_compact(p: KvmParams, K, V, set_start, pivot, out_len, K_out, V_out, out_size, ws, stream=None) -> None:

@@ -70,6 +70,7 @@ struct Workspace {
     int32_t* set_start; // [U,cap+1]
     int32_t* set_id;    // [U,S]
     float* merge_part;  // partial sums of sets that cross token tiles
+    float* attend_part; // per-chunk online-softmax states of the decode-step attention
     size_t bytes;
 };
 
@@ -84,6 +85,7 @@ Workspace carve(const Dims& d, void* base) {
     w.set_start = (int32_t*)take((size_t)d.U * (d.cap + 1) * sizeof(int32_t));
     w.set_id = (int32_t*)take((size_t)d.U * d.S * sizeof(int32_t));
     w.merge_part = (float*)take(merge_scratch_floats(d) * sizeof(float));
+    w.attend_part = (float*)take(attend_scratch_floats(d) * sizeof(float));
     w.bytes = off;
     return w;
 }
@@ -196,6 +198,39 @@ int kvm_layer_ratio(const kvm_params* p, const void* K, float* ratio, float* sim
     float* sim = sim_out ? sim_out : w.sim;
     if (launch_similarity(d, K, sim, st) != cudaSuccess) return KVM_E_CUDA;
     return launch_set_ratio(d, sim, ratio, st) == cudaSuccess ? KVM_OK : KVM_E_CUDA;
+}
+
+int kvm_attend(const kvm_params* p, const void* q, const void* K, const void* V, int32_t rows, const int32_t* len,
+               float* out, void* ws, size_t ws_bytes, void* cuda_stream) {
+    Dims d;
+    int rc = derive(p, d);
+    if (rc != KVM_OK) return rc;
+    if (!q || !K || !V || !out) return KVM_E_NULL;
+    if (rows < 1 || rows > d.S) return KVM_E_SHAPE;
+    if (misaligned(q) || misaligned(K) || misaligned(V) || misaligned(out)) return KVM_E_ALIGN;
+    Workspace w;
+    if ((rc = check_ws(d, ws, ws_bytes, w)) != KVM_OK) return rc;
+    return launch_attend(d, q, K, V, rows, len, out, w.attend_part, (cudaStream_t)cuda_stream) == cudaSuccess
+               ? KVM_OK
+               : KVM_E_CUDA;
+}
+
+int kvm_output_perturbation(const kvm_params* p, const void* q, const void* K, const void* V, const void* K_c,
+                            const void* V_c, const int32_t* len_c, float* out_full, float* out_comp, float* err,
+                            float* ref, void* ws, size_t ws_bytes, void* cuda_stream) {
+    Dims d;
+    int rc = derive(p, d);
+    if (rc != KVM_OK) return rc;
+    if (!q || !K || !V || !K_c || !V_c || !len_c || !out_full || !out_comp || !err || !ref) return KVM_E_NULL;
+    if (misaligned(q) || misaligned(K) || misaligned(V) || misaligned(K_c) || misaligned(V_c) ||
+        misaligned(out_full) || misaligned(out_comp))
+        return KVM_E_ALIGN;
+    Workspace w;
+    if ((rc = check_ws(d, ws, ws_bytes, w)) != KVM_OK) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (launch_attend(d, q, K, V, d.S, nullptr, out_full, w.attend_part, st) != cudaSuccess) return KVM_E_CUDA;
+    if (launch_attend(d, q, K_c, V_c, d.cap, len_c, out_comp, w.attend_part, st) != cudaSuccess) return KVM_E_CUDA;
+    return launch_perturbation(d, out_full, out_comp, err, ref, st) == cudaSuccess ? KVM_OK : KVM_E_CUDA;
 }
 
 int kvm_merge_compact(const kvm_params* p, const void* K, const void* V, const int32_t* set_start,
@@ -349,6 +384,7 @@ int kvm_score_static(const kvm_params* p, const void* Q, const void* K, float* s
     w.set_start = nullptr;
     w.set_id = nullptr;
     w.merge_part = nullptr;
+    w.attend_part = nullptr;
     w.bytes = sizeof(g_static_score_scratch);
     return run_score(d, Q, K, nullptr, scores, w, nullptr, st) == cudaSuccess ? KVM_OK : KVM_E_CUDA;
 }

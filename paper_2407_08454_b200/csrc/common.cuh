@@ -72,4 +72,12 @@ cudaError_t launch_gather(const Dims& d, const void* K, const void* V, const int
                           const int32_t* pivot, const int32_t* out_len, void* K_out, void* V_out, int32_t* out_size,
                           cudaStream_t st);
 
+// Decode-step attention over a ragged cache and the full-vs-compressed output difference.
+int attend_splits(int rows);
+size_t attend_scratch_floats(const Dims& d);
+cudaError_t launch_attend(const Dims& d, const void* q, const void* K, const void* V, int rows, const int32_t* len,
+                          float* out, float* part, cudaStream_t st);
+cudaError_t launch_perturbation(const Dims& d, const float* O, const float* Os, float* err, float* ref,
+                                cudaStream_t st);
+
 }  // namespace kvm
