@@ -16,7 +16,10 @@ namespace kvm {
 namespace {
 
 constexpr int ATT_NT = 256;
-constexpr int ATT_CHUNK = 128;
+#ifndef KVM_ATT_CHUNK
+#define KVM_ATT_CHUNK 256
+#endif
+constexpr int ATT_CHUNK = KVM_ATT_CHUNK;    // cache rows per block
 constexpr float LOG2E = 1.4426950408889634f;
 
 // Weight of a partial state with maximum m when the overall maximum is M (an empty state has m = -inf).
@@ -48,23 +51,53 @@ __global__ void __launch_bounds__(ATT_NT) attend_partial_kernel(const T* __restr
     float m = -INFINITY, l = 0.f, acc[N];
 #pragma unroll
     for (int e = 0; e < N; ++e) acc[e] = 0.f;
-    for (int r = r0 + grp; r < r1; r += NGRP) {
-        const uint4 kraw = ldg16(Ku + (size_t)r * D + lane * N);
-        const uint4 vraw = ldg16(Vu + (size_t)r * D + lane * N);
-        float kf[N], vf[N];
-        Vec<T>::unpack(kraw, kf);
-        float dot = 0.f;
+    // RPI rows per iteration: their loads are independent and in flight together; one rescale per iteration
+#ifndef KVM_ATT_RPI
+#define KVM_ATT_RPI 4
+#endif
+    constexpr int RPI = KVM_ATT_RPI;
+    for (int r = r0 + grp * RPI; r < r1; r += NGRP * RPI) {
+        uint4 kraw[RPI], vraw[RPI];
 #pragma unroll
-        for (int e = 0; e < N; ++e) dot = fmaf(qf[e], kf[e], dot);
+        for (int i = 0; i < RPI; ++i) {
+            const int ri = min(r + i, r1 - 1);                   // clamped rows are loaded but given no weight
+            kraw[i] = ldg16(Ku + (size_t)ri * D + lane * N);
+            vraw[i] = ldg16(Vu + (size_t)ri * D + lane * N);
+        }
+        float s[RPI];
 #pragma unroll
-        for (int off = 1; off < LPR; off <<= 1) dot += __shfl_xor_sync(gmask, dot, off);
-        const float s = dot * scale_log2e;
-        const float mn = fmaxf(m, s);
-        const float corr = exp2f(m - mn), pj = exp2f(s - mn);     // first row: exp2(-inf) = 0
-        l = fmaf(l, corr, pj);
-        Vec<T>::unpack(vraw, vf);
+        for (int i = 0; i < RPI; ++i) {
+            float kf[N];
+            Vec<T>::unpack(kraw[i], kf);
+            float dot = 0.f;
 #pragma unroll
-        for (int e = 0; e < N; ++e) acc[e] = fmaf(acc[e], corr, pj * vf[e]);
+            for (int e = 0; e < N; ++e) dot = fmaf(qf[e], kf[e], dot);
+            s[i] = dot;
+        }
+#pragma unroll
+        for (int off = 1; off < LPR; off <<= 1) {
+#pragma unroll
+            for (int i = 0; i < RPI; ++i) s[i] += __shfl_xor_sync(gmask, s[i], off);
+        }
+        float mn = m;
+#pragma unroll
+        for (int i = 0; i < RPI; ++i) {
+            s[i] = (r + i < r1) ? s[i] * scale_log2e : -INFINITY;
+            mn = fmaxf(mn, s[i]);
+        }
+        const float corr = exp2f(m - mn);                        // first iteration: exp2(-inf) = 0
+        l *= corr;
+#pragma unroll
+        for (int e = 0; e < N; ++e) acc[e] *= corr;
+#pragma unroll
+        for (int i = 0; i < RPI; ++i) {
+            const float pj = exp2f(s[i] - mn);                   // 0 for a clamped row
+            float vf[N];
+            Vec<T>::unpack(vraw[i], vf);
+            l += pj;
+#pragma unroll
+            for (int e = 0; e < N; ++e) acc[e] = fmaf(pj, vf[e], acc[e]);
+        }
         m = mn;
     }
     if (lane == 0) { sm_m[grp] = m; sm_l[grp] = l; }
