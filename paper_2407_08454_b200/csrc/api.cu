@@ -100,10 +100,17 @@ int check_ws(const Dims& d, void* ws, size_t ws_bytes, Workspace& w) {
     return KVM_OK;
 }
 
+// sim_out (nullable): where the neighbour-key similarities are wanted.  *sim_done tells whether the score
+// step produced them on the side (bf16 row pass) or the caller still has to launch the similarity kernel.
 cudaError_t run_score(const Dims& d, const void* Q, const void* K, const float* lse_in, float* scores,
-                      const Workspace& w, kvm_stats* stats, cudaStream_t st) {
+                      const Workspace& w, kvm_stats* stats, cudaStream_t st, float* sim_out = nullptr,
+                      bool* sim_done = nullptr) {
     // bf16: tensor cores (tcgen05); fp32: plain FMA, since tensor-core input rounding cannot hold the score tolerance
-    if (d.dtype == KVM_BF16) return launch_score_tc(d, Q, K, lse_in, w.lse, scores, stats, st);
+    if (d.dtype == KVM_BF16) {
+        if (sim_done) *sim_done = sim_out && !lse_in;
+        return launch_score_tc(d, Q, K, lse_in, w.lse, scores, stats, st, sim_out);
+    }
+    if (sim_done) *sim_done = false;
     return launch_score_simt(d, Q, K, lse_in, w.lse, scores, st);
 }
 
@@ -268,8 +275,11 @@ int kvm_compress(const kvm_params* p, const void* Q, const void* K, const void* 
     if ((rc = check_ws(d, ws, ws_bytes, w)) != KVM_OK) return rc;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     float* scores = scores_out ? scores_out : w.scores;
-    if (run_score(d, Q, K, nullptr, scores, w, stats, st) != cudaSuccess) return KVM_E_CUDA;
-    if (d.set_rule == KVM_SETS_ADJACENT)
+    const bool want_sim = d.set_rule == KVM_SETS_ADJACENT;
+    bool sim_done = false;
+    if (run_score(d, Q, K, nullptr, scores, w, stats, st, want_sim ? w.sim : nullptr, &sim_done) != cudaSuccess)
+        return KVM_E_CUDA;
+    if (want_sim && !sim_done)
         if (launch_similarity(d, K, w.sim, st) != cudaSuccess) return KVM_E_CUDA;
     if (launch_segment(d, scores, w.sim, w.set_id, w.set_start, out_pos, out_len, stats, st) != cudaSuccess)
         return KVM_E_CUDA;

@@ -36,7 +36,7 @@
 // tensor memory is freed and the kernel returns.
 #include <cuda.h>
 
-#include "common.cuh"
+#include "similarity_core.cuh"
 
 namespace kvm {
 namespace {
@@ -50,7 +50,9 @@ constexpr int PCH = 16;              // channels of the lse side tensor (one K =
 constexpr uint32_t PTILE_BYTES = TILE * PCH * 2;   // 4 KB: 128 rows x 32 B
 constexpr int NEPI_WARPS = 16;          // 4 TMEM lane quarters x 4 column quarters
 constexpr int QCOLS = TILE / 4;          // accumulator columns per epilogue warp
-constexpr int NTHREADS = (NEPI_WARPS + 2) * 32;
+constexpr int NSIM_WARPS = 2;           // row pass only: neighbour-key similarities on the side
+constexpr int SIM_RUN = 8;              // consecutive tokens per lane group and round trip
+constexpr int NTHREADS = (NEPI_WARPS + 2 + NSIM_WARPS) * 32;
 constexpr long long WAIT_LIMIT_CLOCKS = 4000000000ll;   // ~2 s of SM clocks: a longer wait is reported, not endured
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float LN2 = 0.6931471805599453f;
@@ -310,7 +312,7 @@ __global__ void __launch_bounds__(NTHREADS, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ CUtensorMap map_p, __nv_bfloat16* __restrict__ lsep_out,
                 float* __restrict__ scores, kvm_stats* stats, int pass, int B, int Hq, int Hkv, int S,
-                float scale2) {
+                float scale2, const __nv_bfloat16* __restrict__ Ksim, float* __restrict__ sim_out) {
     extern __shared__ uint8_t smem_raw[];
     constexpr uint32_t CHUNK_BYTES = TILE * 128;            // one [128 rows x 64 bf16] TMA box
     constexpr uint32_t TILE_BYTES = KCH * CHUNK_BYTES;      // an A tile: [KCH][128 rows][128 B]
@@ -442,6 +444,25 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     umma_commit(&sh.bar.acc_full[as]);     // accumulator ready for the epilogue
                 }
                 if (ok) umma_commit(&sh.bar.empty_a[ab]);  // A tile reusable
+            }
+        }
+    } else if (warp >= NEPI_WARPS + 2) {
+        // ============================== similarity on the side ==============================
+        // Eq. 2 needs nothing but K, and the epilogue warps leave issue slots and memory bandwidth unused:
+        // the key rows are dealt to these warps of all CTAs in runs of SIM_RUN tokens.
+        if (sim_out) {
+            constexpr int D = KCH * KCHUNK, LPR = D / 8, GPW = 32 / LPR;
+            const int runs = (S + SIM_RUN - 1) / SIM_RUN;
+            const long long n_runs = (long long)B * Hkv * runs;
+            const int gl = lane % LPR, gbase = lane / LPR * LPR;
+            const unsigned gmask = (LPR == 32) ? 0xffffffffu : (((1u << LPR) - 1u) << gbase);
+            const long long stride = (long long)gridDim.x * NSIM_WARPS * GPW;
+            for (long long g = ((long long)blockIdx.x * NSIM_WARPS + (warp - NEPI_WARPS - 2)) * GPW + lane / LPR;
+                 g < n_runs; g += stride) {
+                const long long u = g / runs;
+                const int j0 = (int)(g % runs) * SIM_RUN;
+                simcore::run<__nv_bfloat16, D, SIM_RUN>(Ksim + (size_t)u * S * D, sim_out + (size_t)u * S, j0,
+                                                        min(j0 + SIM_RUN, S), gl, gbase, gmask);
             }
         }
     } else {
@@ -646,7 +667,8 @@ __global__ void __launch_bounds__(256) lse_split_kernel(const float* __restrict_
 
 template <int KCH>
 cudaError_t launch_t(const Dims& d, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mp,
-                     const float* lse_in, __nv_bfloat16* side, float* scores, kvm_stats* stats, cudaStream_t st) {
+                     const float* lse_in, __nv_bfloat16* side, float* scores, kvm_stats* stats, cudaStream_t st,
+                     const __nv_bfloat16* Ksim, float* sim_out) {
     const size_t smem = 1024 + (size_t)(2 + 2 * NSTAGE) * KCH * TILE * 128 + (size_t)(2 * NSTAGE + 1) * PTILE_BYTES +
                         sizeof(Shared);
     cudaError_t e = cudaFuncSetAttribute(score_tc_kernel<KCH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -660,7 +682,7 @@ cudaError_t launch_t(const Dims& d, const CUtensorMap& mq, const CUtensorMap& mk
         const long long items = (long long)d.B * d.Hq * T;
         const int grid = (int)(items < sms ? items : sms);
         score_tc_kernel<KCH><<<grid, NTHREADS, smem, st>>>(mq, mk, mp, side, nullptr, stats, 1, d.B, d.Hq, d.Hkv, d.S,
-                                                          scale2);
+                                                          scale2, Ksim, sim_out);
     } else {
         const long long rows = (long long)d.B * d.Hq * d.S;
         lse_split_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(lse_in, side, rows, -LOG2E / scale2);
@@ -669,7 +691,7 @@ cudaError_t launch_t(const Dims& d, const CUtensorMap& mq, const CUtensorMap& mk
     const long long items = (long long)d.U * T;
     const int grid = (int)(items < sms ? items : sms);
     score_tc_kernel<KCH><<<grid, NTHREADS, smem, st>>>(mq, mk, mp, nullptr, scores, stats, 2, d.B, d.Hq, d.Hkv, d.S,
-                                                      scale2);
+                                                      scale2, nullptr, nullptr);
     return cudaGetLastError();
 }
 
@@ -678,15 +700,18 @@ cudaError_t launch_t(const Dims& d, const CUtensorMap& mq, const CUtensorMap& mk
 // Bytes of scratch per query row that the tensor-core path needs (the lse side tensor).
 size_t score_tc_scratch_bytes_per_row() { return (size_t)PCH * 2; }
 
+// sim_out (nullable): when given and the row pass runs (no lse_in), that pass also writes the neighbour-key
+// similarities [U,S] there, so the caller needs no similarity kernel.
 cudaError_t launch_score_tc(const Dims& d, const void* Q, const void* K, const float* lse_in, float* lse_ws,
-                            float* scores, kvm_stats* stats, cudaStream_t st) {
+                            float* scores, kvm_stats* stats, cudaStream_t st, float* sim_out) {
     CUtensorMap mq, mk, mp;
     __nv_bfloat16* side = reinterpret_cast<__nv_bfloat16*>(lse_ws);
     if (!make_map(&mq, Q, d.B * d.Hq, d.S, d.D) || !make_map(&mk, K, d.B * d.Hkv, d.S, d.D) ||
         !make_map_side(&mp, side, d.B * d.Hq, d.S))
         return cudaErrorNotSupported;
-    return d.D == 128 ? launch_t<2>(d, mq, mk, mp, lse_in, side, scores, stats, st)
-                      : launch_t<1>(d, mq, mk, mp, lse_in, side, scores, stats, st);
+    const __nv_bfloat16* Ks = reinterpret_cast<const __nv_bfloat16*>(K);
+    return d.D == 128 ? launch_t<2>(d, mq, mk, mp, lse_in, side, scores, stats, st, Ks, sim_out)
+                      : launch_t<1>(d, mq, mk, mp, lse_in, side, scores, stats, st, Ks, sim_out);
 }
 
 }  // namespace kvm
