@@ -19,7 +19,8 @@
  *   - Unless a parameter says "host", tensor pointers are DEVICE pointers owned by
  *     the caller, contiguous row-major in the stated shape and 16-byte aligned.
  *     Inputs are never written.
- *   - The library allocates no memory and keeps no state between calls.  Scratch
+ *   - The library allocates no device memory and, kvm_compress_host's streams
+ *     aside, keeps no state between calls.  Scratch
  *     space is the caller's `ws` buffer of at least kvm_workspace_bytes() bytes;
  *     its contents are undefined afterwards.  Calls that share a workspace must
  *     be ordered on one stream.
@@ -187,8 +188,14 @@ int kvm_compress(const kvm_params* p, const void* Q, const void* K, const void* 
  * makes the copies asynchronous).  Q, K, V, K_out, V_out, out_len, out_pos are
  * host pointers with the shapes of kvm_compress; `dev` is a caller-owned device
  * buffer of at least kvm_host_staging_bytes() bytes that holds the staged tensors
- * and the workspace.  Copies in, compresses, copies all cap rows out; everything
- * is enqueued on the stream and the caller synchronises before reading.
+ * and the workspace.  Copies in, compresses, copies all cap rows out.  The layer
+ * is cut into groups of units that flow through a three-stage pipeline (copy in
+ * on `cuda_stream`, kernels and copy out on two streams of the library's own), so
+ * that the copies in both directions overlap each other and the kernels;
+ * `cuda_stream` waits for the last copy out, and the caller synchronises it before
+ * reading.  The first call on a device creates the two streams and a handful of
+ * events, which live until the process exits (the one piece of state the library
+ * keeps); calls are serialised by a host mutex while they enqueue.
  */
 int kvm_host_staging_bytes(const kvm_params* p, size_t* bytes);
 int kvm_compress_host(const kvm_params* p, const void* Q, const void* K, const void* V,

@@ -1,7 +1,9 @@
 // C ABI of the kvm library: host-side validation, workspace carving, dispatch.
-// All checks run before anything is enqueued; nothing here allocates or synchronises.
+// All checks run before anything is enqueued; nothing here allocates device memory or synchronises.
 #include <math.h>
 #include <string.h>
+
+#include <mutex>
 
 #include "common.cuh"
 
@@ -309,6 +311,40 @@ int kvm_host_staging_bytes(const kvm_params* p, size_t* bytes) {
     return KVM_OK;
 }
 
+// Streams and events of kvm_compress_host's copy/compute pipeline: created once per device on first use,
+// kept until the process exits.
+namespace {
+
+constexpr int kHostChunksMax = 8;
+constexpr int kPipeDevices = 64;
+
+struct HostPipe {
+    bool ready = false;
+    cudaStream_t compute = nullptr, d2h = nullptr;
+    cudaEvent_t start = nullptr, end = nullptr, h2d[kHostChunksMax] = {}, done[kHostChunksMax] = {};
+};
+HostPipe g_pipe[kPipeDevices];
+std::mutex g_pipe_mu;      // held while a call enqueues: calls on one device share the events
+
+HostPipe* host_pipe_for_current_device() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kPipeDevices) return nullptr;
+    HostPipe& hp = g_pipe[dev];
+    if (hp.ready) return &hp;
+    bool ok = cudaStreamCreateWithFlags(&hp.compute, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&hp.d2h, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&hp.end, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; ok && i < kHostChunksMax; ++i)
+        ok = cudaEventCreateWithFlags(&hp.h2d[i], cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&hp.done[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) return nullptr;
+    hp.ready = true;
+    return &hp;
+}
+
+}  // namespace
+
 int kvm_compress_host(const kvm_params* p, const void* Q, const void* K, const void* V, void* K_out, void* V_out,
                       int32_t* out_len, int32_t* out_pos, void* dev, size_t dev_bytes, void* cuda_stream) {
     Dims d;
@@ -320,26 +356,54 @@ int kvm_compress_host(const kvm_params* p, const void* Q, const void* K, const v
     if (!dev || dev_bytes < need) return KVM_E_WORKSPACE;
     if (misaligned(dev)) return KVM_E_ALIGN;
     const size_t e = d.dtype == KVM_BF16 ? 2 : 4;
-    const size_t nQ = (size_t)d.B * d.Hq * d.S * d.D * e, nK = (size_t)d.U * d.S * d.D * e;
-    const size_t nO = (size_t)d.U * d.cap * d.D * e, nL = (size_t)d.U * sizeof(int32_t);
-    const size_t nP = (size_t)d.U * d.cap * sizeof(int32_t);
+    const size_t rowQ = (size_t)d.G * d.S * d.D * e, rowK = (size_t)d.S * d.D * e;       // bytes per unit
+    const size_t rowO = (size_t)d.cap * d.D * e, rowP = (size_t)d.cap * sizeof(int32_t);
     char* b = (char*)dev;
     size_t off = 0;
     auto take = [&](size_t n) { char* q = b + off; off += align_up(n); return q; };
-    char* dQ = take(nQ); char* dK = take(nK); char* dV = take(nK);
-    char* dKo = take(nO); char* dVo = take(nO); char* dL = take(nL); char* dP = take(nP);
+    char* dQ = take(rowQ * d.U); char* dK = take(rowK * d.U); char* dV = take(rowK * d.U);
+    char* dKo = take(rowO * d.U); char* dVo = take(rowO * d.U);
+    char* dL = take((size_t)d.U * sizeof(int32_t)); char* dP = take(rowP * d.U);
     char* ws = b + off;
+    const size_t ws_bytes = dev_bytes - off;
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    if (cudaMemcpyAsync(dQ, Q, nQ, cudaMemcpyHostToDevice, st) != cudaSuccess) return KVM_E_CUDA;
-    if (cudaMemcpyAsync(dK, K, nK, cudaMemcpyHostToDevice, st) != cudaSuccess) return KVM_E_CUDA;
-    if (cudaMemcpyAsync(dV, V, nK, cudaMemcpyHostToDevice, st) != cudaSuccess) return KVM_E_CUDA;
-    rc = kvm_compress(p, dQ, dK, dV, dKo, dVo, (int32_t*)dL, (int32_t*)dP, nullptr, nullptr, ws, dev_bytes - off,
-                      cuda_stream);
-    if (rc != KVM_OK) return rc;
-    if (cudaMemcpyAsync(K_out, dKo, nO, cudaMemcpyDeviceToHost, st) != cudaSuccess) return KVM_E_CUDA;
-    if (cudaMemcpyAsync(V_out, dVo, nO, cudaMemcpyDeviceToHost, st) != cudaSuccess) return KVM_E_CUDA;
-    if (cudaMemcpyAsync(out_len, dL, nL, cudaMemcpyDeviceToHost, st) != cudaSuccess) return KVM_E_CUDA;
-    if (cudaMemcpyAsync(out_pos, dP, nP, cudaMemcpyDeviceToHost, st) != cudaSuccess) return KVM_E_CUDA;
+
+    // Units are independent and contiguous in every tensor, so the layer is cut into groups of units and
+    // the three stages run as a pipeline: host-to-device copies on the caller's stream, kernels on a second
+    // stream, device-to-host copies on a third.  The caller's stream waits for the last copy out.
+    std::lock_guard<std::mutex> lock(g_pipe_mu);
+    HostPipe* hp = host_pipe_for_current_device();
+    if (!hp) return KVM_E_CUDA;
+    const int nch = d.U < kHostChunksMax ? d.U : kHostChunksMax;
+    const int per = (d.U + nch - 1) / nch;
+    auto ok = [](cudaError_t err) { return err == cudaSuccess; };
+    if (!ok(cudaEventRecord(hp->start, st)) || !ok(cudaStreamWaitEvent(hp->compute, hp->start, 0)) ||
+        !ok(cudaStreamWaitEvent(hp->d2h, hp->start, 0)))
+        return KVM_E_CUDA;
+    for (int c = 0, u0 = 0; u0 < d.U; ++c, u0 += per) {
+        const int nu = (d.U - u0 < per) ? d.U - u0 : per;
+        kvm_params pc = *p;                      // the group as a layer of its own: one batch entry, nu KV heads
+        pc.batch = 1;
+        pc.n_kv_heads = nu;
+        pc.n_q_heads = nu * d.G;
+        if (pc.pivot_key) pc.pivot_key += (size_t)u0 * d.S;
+        if (!ok(cudaMemcpyAsync(dQ + rowQ * u0, (const char*)Q + rowQ * u0, rowQ * nu, cudaMemcpyHostToDevice, st)) ||
+            !ok(cudaMemcpyAsync(dK + rowK * u0, (const char*)K + rowK * u0, rowK * nu, cudaMemcpyHostToDevice, st)) ||
+            !ok(cudaMemcpyAsync(dV + rowK * u0, (const char*)V + rowK * u0, rowK * nu, cudaMemcpyHostToDevice, st)) ||
+            !ok(cudaEventRecord(hp->h2d[c], st)) || !ok(cudaStreamWaitEvent(hp->compute, hp->h2d[c], 0)))
+            return KVM_E_CUDA;
+        rc = kvm_compress(&pc, dQ + rowQ * u0, dK + rowK * u0, dV + rowK * u0, dKo + rowO * u0, dVo + rowO * u0,
+                          (int32_t*)dL + u0, (int32_t*)(dP + rowP * u0), nullptr, nullptr, ws, ws_bytes, hp->compute);
+        if (rc != KVM_OK) return rc;
+        if (!ok(cudaEventRecord(hp->done[c], hp->compute)) || !ok(cudaStreamWaitEvent(hp->d2h, hp->done[c], 0)) ||
+            !ok(cudaMemcpyAsync((char*)K_out + rowO * u0, dKo + rowO * u0, rowO * nu, cudaMemcpyDeviceToHost, hp->d2h)) ||
+            !ok(cudaMemcpyAsync((char*)V_out + rowO * u0, dVo + rowO * u0, rowO * nu, cudaMemcpyDeviceToHost, hp->d2h)) ||
+            !ok(cudaMemcpyAsync(out_len + u0, (int32_t*)dL + u0, (size_t)nu * sizeof(int32_t), cudaMemcpyDeviceToHost,
+                                hp->d2h)) ||
+            !ok(cudaMemcpyAsync((char*)out_pos + rowP * u0, dP + rowP * u0, rowP * nu, cudaMemcpyDeviceToHost, hp->d2h)))
+            return KVM_E_CUDA;
+    }
+    if (!ok(cudaEventRecord(hp->end, hp->d2h)) || !ok(cudaStreamWaitEvent(st, hp->end, 0))) return KVM_E_CUDA;
     return KVM_OK;
 }
 

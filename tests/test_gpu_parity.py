@@ -140,3 +140,40 @@ def test_compress_is_reproducible_bit_for_bit():
     a, b = run_gpu(case), run_gpu(case)
     for f in ("c_scores", "c_out_len", "c_out_pos", "c_K_out", "c_V_out"):
         assert np.array_equal(getattr(a, f), getattr(b, f)), f
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,S,D,dtype", [
+    (1, 4, 4, 512, 64, torch.float32),
+    (2, 6, 3, 700, 128, torch.bfloat16),      # 6 units: one per group
+    (5, 4, 2, 300, 128, torch.bfloat16),      # 10 units: groups of 2, GQA
+    (1, 2, 1, 256, 64, torch.bfloat16),       # a single unit
+])
+def test_host_entry_point_equals_the_device_path(B, Hq, Hkv, S, D, dtype):
+    cfg = si.CONFIGS["C1"].scaled(seq=S, head_dim=D, n_q_heads=Hq, n_kv_heads=Hkv, batch=B,
+                                  dtype="bf16" if dtype == torch.bfloat16 else "f32", seed=300 + S)
+    d = si.make_layer(cfg)
+    key = torch.rand(B, Hkv, S)
+    for rules in (dict(), dict(pivot_rule=kvm.KVM_PIVOT_KEY, pivot_key=key.cuda())):
+        p = kvm.make_params(B, Hq, Hkv, S, D, dtype, budget=0.5, **rules)
+        comp = kvm.Compressor(p)
+        r = comp(d["Q"].cuda(), d["K"].cuda(), d["V"].cuda())
+        torch.cuda.synchronize()
+        cap = comp.cap
+        pin = {k: v.pin_memory() for k, v in d.items()}
+        hK = torch.full((B, Hkv, cap, D), 768.0, dtype=dtype).pin_memory()
+        hV = torch.full_like(hK, 768.0).pin_memory()
+        hlen = torch.full((B * Hkv,), -7, dtype=torch.int32).pin_memory()
+        hpos = torch.full((B * Hkv, cap), -7, dtype=torch.int32).pin_memory()
+        stage = torch.empty(kvm.kvm_host_staging_bytes(p), dtype=torch.uint8, device="cuda")
+        side = torch.cuda.Stream()
+        for stream in (None, side, None):      # repeated calls reuse the pipeline's events
+            hlen.fill_(-7)
+            with torch.cuda.stream(side if stream is not None else torch.cuda.current_stream()):
+                kvm.kvm_compress_host(p, pin["Q"], pin["K"], pin["V"], hK, hV, hlen, hpos, stage, stream)
+            (stream or torch.cuda.current_stream()).synchronize()
+            assert torch.equal(hlen, r.out_len.cpu().view(-1))
+            for u in range(B * Hkv):
+                n = int(hlen[u])
+                assert torch.equal(hpos[u, :n], r.out_pos.cpu().view(B * Hkv, cap)[u, :n])
+                assert torch.equal(hK.view(B * Hkv, cap, D)[u, :n], r.K_out.cpu().view(B * Hkv, cap, D)[u, :n])
+                assert torch.equal(hV.view(B * Hkv, cap, D)[u, :n], r.V_out.cpu().view(B * Hkv, cap, D)[u, :n])
