@@ -227,7 +227,7 @@ def main():
     # ---- per-kernel timing (same launches, event pairs around each public step)
     b0 = bufs[0]
     scores = torch.empty(cfg.batch, cfg.n_kv_heads, cfg.seq, device=dev)
-    lse = torch.empty(cfg.batch, cfg.n_q_heads, cfg.seq, device=dev)
+    lses = [torch.empty(cfg.batch, cfg.n_q_heads, cfg.seq, device=dev) for _ in range(N_BUFFERS)]
     set_start = torch.empty(cfg.batch, cfg.n_kv_heads, comp.cap + 1, dtype=torch.int32, device=dev)
 
     def timed(fn, reps):
@@ -246,16 +246,18 @@ def main():
     ws = comp.ws
     t_score = timed(lambda i: kvm.kvm_score(p, bufs[i % N_BUFFERS]["Q"], bufs[i % N_BUFFERS]["K"], None, scores, ws,
                                             stream), reps)
-    # natural-log row log-sum-exp for buffer 0 (plain torch, outside every timed region), so that the
-    # column pass can be timed alone through the public lse_in argument
+    # natural-log row log-sum-exp of every input set (plain torch, outside every timed region), so that the
+    # column pass can be timed alone through the public lse_in argument, on rotating inputs like the rest
     mask = torch.ones(cfg.seq, cfg.seq, dtype=torch.bool, device=dev).tril()
     G = cfg.n_q_heads // cfg.n_kv_heads
-    for bb in range(cfg.batch):
-        for h in range(cfg.n_q_heads):
-            logits = (b0["Q"][bb, h].float() @ b0["K"][bb, h // G].float().T) / math.sqrt(cfg.head_dim)
-            lse[bb, h] = torch.logsumexp(logits.masked_fill(~mask, float("-inf")), dim=-1)
+    for bi, lse_b in zip(bufs, lses):
+        for bb in range(cfg.batch):
+            for h in range(cfg.n_q_heads):
+                logits = (bi["Q"][bb, h].float() @ bi["K"][bb, h // G].float().T) / math.sqrt(cfg.head_dim)
+                lse_b[bb, h] = torch.logsumexp(logits.masked_fill(~mask, float("-inf")), dim=-1)
     del mask, logits
-    t_colsum = timed(lambda i: kvm.kvm_score(p, b0["Q"], b0["K"], lse, scores, ws, stream), reps)
+    t_colsum = timed(lambda i: kvm.kvm_score(p, bufs[i % N_BUFFERS]["Q"], bufs[i % N_BUFFERS]["K"],
+                                             lses[i % N_BUFFERS], scores, ws, stream), reps)
     t_segment = timed(lambda i: kvm.kvm_segment(p, bufs[i % N_BUFFERS]["K"], scores, None, set_start, comp.out_pos,
                                                 comp.out_len, None, None, ws, stream), reps)
     t_merge = timed(lambda i: kvm.kvm_merge_compact(p, bufs[i % N_BUFFERS]["K"], bufs[i % N_BUFFERS]["V"], set_start,
@@ -305,6 +307,11 @@ def main():
         "compress_eviction_ms": t_compress(params(set_rule=kvm.KVM_SETS_CONSERVED_ONLY, recent_ratio=0.17,
                                                   heavy_ratio=cfg.budget - 0.17)),
     }
+    # the whole path when the prefill attention already supplies the row log-sum-exp
+    extras["compress_with_lse_ms"] = timed(
+        lambda i: kvm.kvm_compress_with_lse(p, bufs[i % N_BUFFERS]["Q"], bufs[i % N_BUFFERS]["K"],
+                                            bufs[i % N_BUFFERS]["V"], lses[i % N_BUFFERS], comp.K_out, comp.V_out,
+                                            comp.out_len, comp.out_pos, None, None, ws, stream), min(reps, 50))
     ratio = torch.empty(U, device=dev)
     extras["layer_ratio_ms"] = timed(lambda i: kvm.kvm_layer_ratio(p, bufs[i % N_BUFFERS]["K"], ratio, None, ws,
                                                                    stream), min(reps, 50))

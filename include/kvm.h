@@ -184,6 +184,16 @@ int kvm_compress(const kvm_params* p, const void* Q, const void* K, const void* 
                  float* scores_out, kvm_stats* stats, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * kvm_compress for callers that already hold the row log-sum-exp of the layer's causal attention (a fused
+ * prefill attention kernel produces it as a by-product): lse_in [batch, n_q_heads, S] fp32, natural log, of
+ * the logits scaled by softmax_scale.  The row pass of the score step is skipped, which halves the score
+ * step's work (Eq. 1 is evaluated once per query-key pair instead of twice).  lse_in NULL = kvm_compress.
+ */
+int kvm_compress_with_lse(const kvm_params* p, const void* Q, const void* K, const void* V, const float* lse_in,
+                          void* K_out, void* V_out, int32_t* out_len, int32_t* out_pos, float* scores_out,
+                          kvm_stats* stats, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
  * kvm_compress for callers whose tensors live in HOST memory (pinned memory
  * makes the copies asynchronous).  Q, K, V, K_out, V_out, out_len, out_pos are
  * host pointers with the shapes of kvm_compress; `dev` is a caller-owned device

@@ -24,6 +24,7 @@ KVM_WEIGHT_GAUSSIAN, KVM_WEIGHT_AVERAGE, KVM_WEIGHT_PIVOT_ONLY = 0, 1, 2
 KVM_SETS_ADJACENT, KVM_SETS_CONSERVED_ONLY = 0, 1
 EXPORTS = (
     "kvm_sizes", "kvm_workspace_bytes", "kvm_score", "kvm_segment", "kvm_merge_compact", "kvm_compress",
+    "kvm_compress_with_lse",
     "kvm_host_staging_bytes", "kvm_compress_host", "kvm_score_static", "kvm_layer_ratio", "kvm_attend",
     "kvm_output_perturbation", "kvm_status_string",
     "kvm_version",
@@ -189,6 +190,14 @@ def kvm_compress(p: KvmParams, Q, K, V, K_out, V_out, out_len, out_pos, scores_o
     _check(lib().kvm_compress(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(K_out), _ptr(V_out), _ptr(out_len),
                               _ptr(out_pos), _ptr(scores_out), _ptr(stats), _ptr(ws),
                               ctypes.c_size_t(ws.numel() * ws.element_size()), _stream(stream)), "kvm_compress")
+
+
+def kvm_compress_with_lse(p: KvmParams, Q, K, V, lse_in, K_out, V_out, out_len, out_pos, scores_out, stats, ws,
+                          stream=None) -> None:
+    _check(lib().kvm_compress_with_lse(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(lse_in), _ptr(K_out),
+                                       _ptr(V_out), _ptr(out_len), _ptr(out_pos), _ptr(scores_out), _ptr(stats),
+                                       _ptr(ws), ctypes.c_size_t(ws.numel() * ws.element_size()), _stream(stream)),
+           "kvm_compress_with_lse")
 
 
 def kvm_compress_host(p: KvmParams, Q, K, V, K_out, V_out, out_len, out_pos, dev, stream=None) -> None:

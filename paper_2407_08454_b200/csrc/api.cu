@@ -109,7 +109,7 @@ cudaError_t run_score(const Dims& d, const void* Q, const void* K, const float* 
                       bool* sim_done = nullptr) {
     // bf16: tensor cores (tcgen05); fp32: plain FMA, since tensor-core input rounding cannot hold the score tolerance
     if (d.dtype == KVM_BF16) {
-        if (sim_done) *sim_done = sim_out && !lse_in;
+        if (sim_done) *sim_done = sim_out != nullptr;
         return launch_score_tc(d, Q, K, lse_in, w.lse, scores, stats, st, sim_out);
     }
     if (sim_done) *sim_done = false;
@@ -266,12 +266,19 @@ int kvm_merge_compact(const kvm_params* p, const void* K, const void* V, const i
 int kvm_compress(const kvm_params* p, const void* Q, const void* K, const void* V, void* K_out, void* V_out,
                  int32_t* out_len, int32_t* out_pos, float* scores_out, kvm_stats* stats, void* ws,
                  size_t ws_bytes, void* cuda_stream) {
+    return kvm_compress_with_lse(p, Q, K, V, nullptr, K_out, V_out, out_len, out_pos, scores_out, stats, ws,
+                                 ws_bytes, cuda_stream);
+}
+
+int kvm_compress_with_lse(const kvm_params* p, const void* Q, const void* K, const void* V, const float* lse_in,
+                          void* K_out, void* V_out, int32_t* out_len, int32_t* out_pos, float* scores_out,
+                          kvm_stats* stats, void* ws, size_t ws_bytes, void* cuda_stream) {
     Dims d;
     int rc = derive(p, d);
     if (rc != KVM_OK) return rc;
     if (!Q || !K || !V || !K_out || !V_out || !out_len || !out_pos) return KVM_E_NULL;
     if (misaligned(Q) || misaligned(K) || misaligned(V) || misaligned(K_out) || misaligned(V_out) ||
-        (scores_out && misaligned(scores_out)))
+        (scores_out && misaligned(scores_out)) || (lse_in && misaligned(lse_in)))
         return KVM_E_ALIGN;
     Workspace w;
     if ((rc = check_ws(d, ws, ws_bytes, w)) != KVM_OK) return rc;
@@ -279,7 +286,7 @@ int kvm_compress(const kvm_params* p, const void* Q, const void* K, const void* 
     float* scores = scores_out ? scores_out : w.scores;
     const bool want_sim = d.set_rule == KVM_SETS_ADJACENT;
     bool sim_done = false;
-    if (run_score(d, Q, K, nullptr, scores, w, stats, st, want_sim ? w.sim : nullptr, &sim_done) != cudaSuccess)
+    if (run_score(d, Q, K, lse_in, scores, w, stats, st, want_sim ? w.sim : nullptr, &sim_done) != cudaSuccess)
         return KVM_E_CUDA;
     if (want_sim && !sim_done)
         if (launch_similarity(d, K, w.sim, st) != cudaSuccess) return KVM_E_CUDA;

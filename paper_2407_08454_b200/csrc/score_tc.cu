@@ -50,7 +50,7 @@ constexpr int PCH = 16;              // channels of the lse side tensor (one K =
 constexpr uint32_t PTILE_BYTES = TILE * PCH * 2;   // 4 KB: 128 rows x 32 B
 constexpr int NEPI_WARPS = 16;          // 4 TMEM lane quarters x 4 column quarters
 constexpr int QCOLS = TILE / 4;          // accumulator columns per epilogue warp
-constexpr int NSIM_WARPS = 2;           // row pass only: neighbour-key similarities on the side
+constexpr int NSIM_WARPS = 2;           // neighbour-key similarities on the side (one of the two passes)
 constexpr int SIM_RUN = 8;              // consecutive tokens per lane group and round trip
 constexpr int NTHREADS = (NEPI_WARPS + 2 + NSIM_WARPS) * 32;
 constexpr long long WAIT_LIMIT_CLOCKS = 4000000000ll;   // ~2 s of SM clocks: a longer wait is reported, not endured
@@ -687,11 +687,12 @@ cudaError_t launch_t(const Dims& d, const CUtensorMap& mq, const CUtensorMap& mk
         const long long rows = (long long)d.B * d.Hq * d.S;
         lse_split_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(lse_in, side, rows, -LOG2E / scale2);
     }
+    const bool sim_in_pass2 = lse_in != nullptr;      // no row pass: the column pass's spare warps do it
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     const long long items = (long long)d.U * T;
     const int grid = (int)(items < sms ? items : sms);
     score_tc_kernel<KCH><<<grid, NTHREADS, smem, st>>>(mq, mk, mp, nullptr, scores, stats, 2, d.B, d.Hq, d.Hkv, d.S,
-                                                      scale2, nullptr, nullptr);
+                                                      scale2, Ksim, sim_in_pass2 ? sim_out : nullptr);
     return cudaGetLastError();
 }
 
@@ -700,8 +701,8 @@ cudaError_t launch_t(const Dims& d, const CUtensorMap& mq, const CUtensorMap& mk
 // Bytes of scratch per query row that the tensor-core path needs (the lse side tensor).
 size_t score_tc_scratch_bytes_per_row() { return (size_t)PCH * 2; }
 
-// sim_out (nullable): when given and the row pass runs (no lse_in), that pass also writes the neighbour-key
-// similarities [U,S] there, so the caller needs no similarity kernel.
+// sim_out (nullable): when given, the spare warps of the row pass (of the column pass when lse_in replaces
+// the row pass) also write the neighbour-key similarities [U,S] there, so the caller needs no similarity kernel.
 cudaError_t launch_score_tc(const Dims& d, const void* Q, const void* K, const float* lse_in, float* lse_ws,
                             float* scores, kvm_stats* stats, cudaStream_t st, float* sim_out) {
     CUtensorMap mq, mk, mp;

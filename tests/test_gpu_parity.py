@@ -94,6 +94,44 @@ def test_lse_in_skips_the_row_pass_and_matches():
     assert score_excess(out.cpu().numpy(), ref) <= 1.0
 
 
+@pytest.mark.parametrize("dtype,S,D", [("bf16", 900, 128), ("f32", 512, 64)])
+def test_compress_with_caller_lse_matches_the_checker(dtype, S, D):
+    from oracle import kvmo
+    from parity import _chain, f32, kv_error, score_excess, KV_TOL
+    cfg = si.CONFIGS["C1"].scaled(seq=S, head_dim=D, n_q_heads=4, n_kv_heads=2, dtype=dtype, seed=11)
+    d = si.make_layer(cfg)
+    case = Case(d["Q"], d["K"], d["V"], budget=0.5)
+    ref, lse = kvmo.scores(d["Q"], d["K"], want_lse=True)
+    p = case.params()
+    comp = kvm.Compressor(p, want_scores=True)
+    Q, K, V = d["Q"].cuda(), d["K"].cuda(), d["V"].cuda()
+    kvm.kvm_compress_with_lse(p, Q, K, V, torch.from_numpy(lse).float().cuda(), comp.K_out, comp.V_out, comp.out_len,
+                              comp.out_pos, comp.scores, None, comp.ws)
+    torch.cuda.synchronize()
+    g_scores = comp.scores.cpu().numpy().reshape(2, S)
+    assert score_excess(g_scores, ref.reshape(2, S)) <= 1.0
+    # the similarities the path used are the similarity kernel's (same code in the score kernel's spare warps)
+    sim = torch.empty(1, 2, S, device="cuda")
+    ratio = torch.empty(2, device="cuda")
+    kvm.kvm_layer_ratio(p, K, ratio, sim, comp.ws)
+    cap, n_r, n_h = kvm.kvm_sizes(p)
+    ch = _chain(case, g_scores.astype(np.float64), sim.cpu().numpy().reshape(2, S).astype(np.float64), cap, n_r, n_h)
+    g_len = comp.out_len.cpu().numpy().reshape(2)
+    assert np.array_equal(g_len, ch["out_len"])
+    g_pos = comp.out_pos.cpu().numpy().reshape(2, cap)
+    rK, rV = kvmo.merge(d["K"][0], d["V"][0], ch["set_start"], ch["pivot"], ch["out_len"], f32(5.0), True)
+    for u in range(2):
+        n = g_len[u]
+        assert np.array_equal(g_pos[u, :n], ch["pivot"][u, :n])
+        assert kv_error(comp.K_out[0, u, :n].float().cpu().numpy(), rK[u, :n]) <= KV_TOL
+        assert kv_error(comp.V_out[0, u, :n].float().cpu().numpy(), rV[u, :n]) <= KV_TOL
+    # and lse_in = NULL is kvm_compress itself
+    a = kvm.Compressor(p)(Q, K, V)
+    b = kvm.Compressor(p)
+    kvm.kvm_compress_with_lse(p, Q, K, V, None, b.K_out, b.V_out, b.out_len, b.out_pos, None, None, b.ws)
+    assert torch.equal(a.out_len, b.out_len) and torch.equal(a.K_out, b.K_out) and torch.equal(a.out_pos, b.out_pos)
+
+
 def test_c1_llama2_7b_layer_full():
     case = _case(si.CONFIGS["C1"])
     g = run_gpu(case)
