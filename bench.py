@@ -390,7 +390,7 @@ def main():
                        "seq_len": cfg.seq, "head_dim": cfg.head_dim, "budget": cfg.budget, "layers_per_step": 1,
                        "l2": f"inputs larger than L2: {N_BUFFERS} rotating layer input sets of 100.7 MB",
                        "parallelism": f"replicas x{world} (independent layers per GPU, no collective)"},
-            "clocks": clk.summary(), "e2e": e2e, "gpu_launches": 6 * args.steps,
+            "clocks": clk.summary(), "e2e": e2e, "gpu_launches": 5 * args.steps,
             "roofline": roofline, "kernels": kernels, "extras": extras,
             "path_roofline": {"roof_ms_per_step": t_roof_ms, "frac": e2e_frac,
                               "note": "slower of 2 score passes at bf16 peak and total bytes at HBM peak"},
