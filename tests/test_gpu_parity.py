@@ -167,6 +167,20 @@ def test_c3_mistral_gqa_32k_layer():
     assert g.cap == 16384
 
 
+def test_maximum_sequence_length():
+    # S = KVM_MAX_SEQ = 65536, one head of 64 channels: the longest sequence the library accepts (512 row tiles,
+    # 64 KB of flags in the segment kernel's shared memory); one more token is refused on the host
+    cfg = si.CONFIGS["C1"].scaled(seq=65536, head_dim=64, n_q_heads=1, n_kv_heads=1, seed=65)
+    case = _case(cfg)
+    g = run_gpu(case)
+    check_invariants_all_units(case, g)
+    rep = check_case(case, g)
+    print("S=65536", rep)
+    with pytest.raises(kvm.KvmError) as e:
+        kvm.kvm_sizes(kvm.make_params(1, 1, 1, 65537, 64, torch.bfloat16))
+    assert e.value.status == -2
+
+
 def test_c4_llama2_13b_layer():
     # batch 8 x 40 heads = 320 units, keys with regime switches (many short sets), 35 % budget
     rng = np.random.default_rng(4)
