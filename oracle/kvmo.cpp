@@ -196,6 +196,49 @@ void kvmo_layer_ratio(int64_t U, int32_t S, double eps, const double* sim, doubl
     }
 }
 
+// Set identification as Section 3.2 words it ("anchor" reading): starting from
+// the last token, a key state gathers the consecutive states before it whose
+// similarity TO IT exceeds eps; the first state that fails (or is conserved, or
+// the start of the sequence) ends the group, and the walk goes on from there.
+// A conserved state is a group of its own.  (Algorithm 1's listing compares
+// neighbours instead; both readings give consecutive, disjoint, covering sets.)
+//   cos(a, b) = <a,b> / (|a||b|), 0 if a norm is 0, computed in fp64.
+// b [U,S] (0/1) = boundary flags (1 at the first token of every group);
+// run (nullable) [U,S] = for EVERY token i, the number of consecutive
+// predecessors whose similarity to k_i exceeds eps, ignoring conserved tokens
+// (the quantity the walk consults at its anchors).
+void kvmo_boundaries_anchor(int64_t U, int32_t S, int32_t D, double eps, const float* K, const uint8_t* keep,
+                            uint8_t* b, int32_t* run) {
+#pragma omp parallel for schedule(static, 1)
+    for (int64_t u = 0; u < U; ++u) {
+        const float* Ku = K + (size_t)u * S * D;
+        const uint8_t* kp = keep + (size_t)u * S;
+        auto cosine = [&](int32_t i, int32_t j) {
+            double dot = 0.0, ni = 0.0, nj = 0.0;
+            for (int32_t t = 0; t < D; ++t) {
+                const double a = Ku[(size_t)i * D + t], c = Ku[(size_t)j * D + t];
+                dot += a * c; ni += a * a; nj += c * c;
+            }
+            return (ni > 0.0 && nj > 0.0) ? dot / (std::sqrt(ni) * std::sqrt(nj)) : 0.0;
+        };
+        if (run)
+            for (int32_t i = 0; i < S; ++i) {
+                int32_t j = i - 1;
+                while (j >= 0 && cosine(i, j) > eps) --j;
+                run[(size_t)u * S + i] = i - 1 - j;
+            }
+        for (int32_t j = 0; j < S; ++j) b[(size_t)u * S + j] = 0;
+        int32_t i = S - 1;
+        while (i >= 0) {
+            int32_t j = i - 1;
+            if (!kp[i])
+                while (j >= 0 && !kp[j] && cosine(i, j) > eps) --j;
+            b[(size_t)u * S + j + 1] = 1;       // the group is tokens j+1 .. i
+            i = j;
+        }
+    }
+}
+
 // Definition 4.1's partition: consecutive, disjoint sets covering the sequence.
 // set_id_j = (number of flags at positions <= j) - 1; set s = [set_start[s], set_start[s+1]).
 // set_id [U,S]; set_start [U,cap+1]; out_len [U].  Entries past out_len are untouched.
@@ -366,7 +409,8 @@ void kvmo_perturbation(int64_t n, int32_t D, const double* O, const double* O_st
 // caller-allocated; cap = C when enforce_budget, else S.
 // Variants (all 0 = the paper's method): pivot_rule 1 = last index of the set,
 // 2 = arg-max of pivot_key [U,S] (iid random numbers give the random-pivot
-// ablation of Section 5.3); weight_rule as in kvmo_merge; set_rule 1 = eviction
+// ablation of Section 5.3); weight_rule as in kvmo_merge; set_rule 2 = the anchor
+// reading of the set identification (kvmo_boundaries_anchor); set_rule 1 = eviction
 // (kvmo_evict; set_id is -1 for dropped tokens, set_start[s] = the kept token).
 void kvmo_compress(int32_t B, int32_t Hq, int32_t Hkv, int32_t S, int32_t D, double scale,
                    int32_t cap, int32_t n_r, int32_t n_h, double eps, double sigma,
@@ -395,7 +439,8 @@ void kvmo_compress(int32_t B, int32_t Hq, int32_t Hkv, int32_t S, int32_t D, dou
         }
         return;
     }
-    kvmo_boundaries(U, S, cap, eps, enforce_budget, sim, keep, b, nullptr);
+    if (set_rule == 2) kvmo_boundaries_anchor(U, S, D, eps, K, keep, b, nullptr);   // no budget rule: cap must be S
+    else kvmo_boundaries(U, S, cap, eps, enforce_budget, sim, keep, b, nullptr);
     kvmo_sets(U, S, cap, b, set_id, set_start, out_len);
     if (pivot_rule == 1) kvmo_pivots_last(U, cap, set_start, out_len, pivot);
     else kvmo_pivots(U, S, cap, pivot_rule == 2 ? pivot_key : scores, set_start, out_len, pivot);

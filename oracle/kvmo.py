@@ -111,6 +111,19 @@ def layer_ratio(sim: np.ndarray, eps: float) -> np.ndarray:
     return out
 
 
+def boundaries_anchor(K, keep_: np.ndarray, eps: float, want_run: bool = False):
+    """Anchor reading of the set identification (Section 3.2): flags [.., S], and the run length of every token."""
+    K = _f32(K)
+    keep_ = np.ascontiguousarray(keep_, dtype=np.uint8)
+    S, D = K.shape[-2:]
+    U = K.size // (S * D)
+    b = np.empty(K.shape[:-1], dtype=np.uint8)
+    run = np.empty(K.shape[:-1], dtype=np.int32) if want_run else None
+    lib().kvmo_boundaries_anchor(ctypes.c_int64(U), ctypes.c_int32(S), ctypes.c_int32(D), ctypes.c_double(eps),
+                                 _p(K), _p(keep_), _p(b), _p(run))
+    return (b, run) if want_run else b
+
+
 def sets(b: np.ndarray, cap: int):
     b = np.ascontiguousarray(b, dtype=np.uint8)
     S = b.shape[-1]
@@ -164,7 +177,7 @@ def evict(keep_: np.ndarray, K, V, cap: int):
 
 PIVOT_MAX_SCORE, PIVOT_LAST, PIVOT_KEY = 0, 1, 2
 WEIGHT_GAUSSIAN, WEIGHT_AVERAGE, WEIGHT_PIVOT_ONLY = 0, 1, 2
-SETS_ADJACENT, SETS_CONSERVED_ONLY = 0, 1
+SETS_ADJACENT, SETS_CONSERVED_ONLY, SETS_ANCHOR = 0, 1, 2
 
 
 def merge(K, V, set_start, pivot, out_len, sigma: float, scale_v: bool = True, want_weights: bool = False,

@@ -175,3 +175,79 @@ def test_layer_ratio_of_wide_ar1_keys_is_a_step_in_rho():
     assert np.abs(sim[0, 1:] - rho).max() < 0.02
     assert kvmo.layer_ratio(sim, rho - 0.05)[0] == 1 / S
     assert kvmo.layer_ratio(sim, rho + 0.05)[0] == 1.0
+
+
+# ---------------------------------------------------------------- anchor reading of the set identification
+def _cos(a, b):
+    a, b = a.astype(np.float64), b.astype(np.float64)
+    na, nb = np.linalg.norm(a), np.linalg.norm(b)
+    return float(a @ b / (na * nb)) if na > 0 and nb > 0 else 0.0
+
+
+def test_anchor_grouping_is_the_unique_partition_with_its_defining_properties():
+    # Walking from the last token, the result is fixed by: every member is similar to its group's LAST token;
+    # the token before a group is not (or is conserved, or does not exist); conserved tokens stand alone.
+    rng = np.random.default_rng(20)
+    for trial in range(20):
+        S, D = int(rng.integers(3, 40)), 3
+        x = np.cumsum(rng.standard_normal((1, S, D)) * 0.35, axis=1).astype(np.float32) + 1.0   # slowly turning keys
+        keep = (rng.random((1, S)) < 0.15).astype(np.uint8)
+        eps = float(rng.uniform(0.5, 0.95))
+        b, run = kvmo.boundaries_anchor(x, keep, eps, want_run=True)
+        assert b[0, 0] == 1
+        starts = np.nonzero(b[0])[0]
+        ends = np.append(starts[1:], S) - 1
+        for lo, hi in zip(starts, ends):
+            if keep[0, lo:hi + 1].any():
+                assert lo == hi
+                continue
+            assert all(_cos(x[0, hi], x[0, j]) > eps for j in range(lo, hi))
+            assert lo == 0 or keep[0, lo - 1] or not (_cos(x[0, hi], x[0, lo - 1]) > eps)
+        for i in range(S):                      # run lengths: brute force over every anchor candidate
+            r = 0
+            while i - 1 - r >= 0 and _cos(x[0, i], x[0, i - 1 - r]) > eps:
+                r += 1
+            assert run[0, i] == r
+
+
+def test_anchor_and_neighbour_readings_differ_exactly_where_they_should():
+    def unit(deg):
+        t = np.deg2rad(np.array(deg, dtype=np.float64))
+        return np.stack([np.cos(t), np.sin(t)], -1)[None].astype(np.float32)
+    none = np.zeros((1, 3), np.uint8)
+    # keys turning by 25 degrees per token: neighbours are similar (cos 25 = 0.906) so Algorithm 1's neighbour
+    # reading chains all three, but token 0 is 50 degrees from the last token (cos 50 = 0.643 < 0.75)
+    K = unit([0, 25, 50])
+    np.testing.assert_array_equal(kvmo.boundaries_anchor(K, none, 0.75)[0], [1, 1, 0])
+    b_adj, _ = kvmo.boundaries(kvmo.similarity(K), none, C=3, eps=0.75)
+    np.testing.assert_array_equal(b_adj[0], [1, 0, 0])
+    # when every state within a neighbour-run is also similar to the run's last state, the readings agree
+    K = unit([0, 5, 10, 80, 85, 170])
+    none = np.zeros((1, 6), np.uint8)
+    b_adj, _ = kvmo.boundaries(kvmo.similarity(K), none, C=6, eps=0.75)
+    np.testing.assert_array_equal(kvmo.boundaries_anchor(K, none, 0.75)[0], b_adj[0])
+    np.testing.assert_array_equal(b_adj[0], [1, 0, 0, 1, 0, 1])
+    # limits: identical keys -> one group; orthogonal keys -> singletons; a conserved token splits the run
+    ident = np.repeat(_rand((1, 1, 8), 21), 9, axis=1)
+    assert kvmo.boundaries_anchor(ident, np.zeros((1, 9), np.uint8), 0.75).sum() == 1
+    assert kvmo.boundaries_anchor(np.eye(8, dtype=np.float32)[None], np.zeros((1, 8), np.uint8), 0.75).sum() == 8
+    keep = np.zeros((1, 9), np.uint8)
+    keep[0, 4] = 1
+    np.testing.assert_array_equal(kvmo.boundaries_anchor(ident, keep, 0.75)[0], [1, 0, 0, 0, 1, 1, 0, 0, 0])
+    # the number of groups never falls when the threshold rises
+    K = np.cumsum(_rand((1, 200, 4), 22) * 0.3, axis=1) + 1.0
+    n = [kvmo.boundaries_anchor(K, np.zeros((1, 200), np.uint8), e).sum() for e in np.linspace(0.0, 0.99, 12)]
+    assert n[0] <= n[-1] and n[-1] > n[0]
+
+
+def test_compress_with_anchor_sets_equals_its_steps():
+    cfg = si.CONFIGS["C0"]
+    d = si.make_layer(cfg)
+    r = kvmo.compress(d["Q"], d["K"], d["V"], 0.50, 0.17, 0.12, enforce_budget=False, set_rule=kvmo.SETS_ANCHOR)
+    b = kvmo.boundaries_anchor(d["K"], r.keep, 0.75)
+    np.testing.assert_array_equal(b, r.b)
+    set_id, st, ol = kvmo.sets(b, cap=cfg.seq)
+    np.testing.assert_array_equal(ol, r.out_len)
+    np.testing.assert_array_equal(kvmo.pivots(r.scores, st, ol), r.pivot)
+    base = kvmo.compress(d["Q"], d["K"], d["V"], 0.50, 0.17, 0.12, enforce_budget=False)
+    assert (r.out_len >= base.out_len).all()        # similarity to the anchor is the stricter requirement here
