@@ -299,7 +299,14 @@ def main():
                                                 comp.out_pos, None, None, ws, stream), min(reps, 50))
 
     key = torch.rand(cfg.batch, cfg.n_kv_heads, cfg.seq, device=dev)
+    p_anchor = params(set_rule=kvm.KVM_SETS_ANCHOR, enforce_budget=0)      # capacity S: its own buffers
+    comp_a = kvm.Compressor(p_anchor, device=dev)
+    t_anchor = timed(lambda i: kvm.kvm_compress(p_anchor, bufs[i % N_BUFFERS]["Q"], bufs[i % N_BUFFERS]["K"],
+                                                bufs[i % N_BUFFERS]["V"], comp_a.K_out, comp_a.V_out, comp_a.out_len,
+                                                comp_a.out_pos, None, None, comp_a.ws, stream), min(reps, 50))
+    del comp_a
     extras = {
+        "compress_anchor_sets_ms": t_anchor,
         "compress_average_last_pivot_ms": t_compress(params(pivot_rule=kvm.KVM_PIVOT_LAST,
                                                             weight_rule=kvm.KVM_WEIGHT_AVERAGE)),
         "compress_keyed_pivot_ms": t_compress(params(pivot_rule=kvm.KVM_PIVOT_KEY, pivot_key=key)),

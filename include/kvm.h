@@ -98,6 +98,12 @@ enum kvm_weight_rule {
 /* Which states reach the output. */
 enum kvm_set_rule {
     KVM_SETS_ADJACENT = 0,       /* Algorithm 1: every token belongs to a merging set */
+    KVM_SETS_ANCHOR = 2,         /* the set identification as Section 3.2 words it: walking from the last token, a
+                                    state gathers the consecutive states before it whose similarity TO IT exceeds
+                                    sim_threshold (Algorithm 1's listing compares neighbours instead).  Conserved
+                                    tokens stand alone.  No budget rule: enforce_budget must be 0 (capacity S), and
+                                    seq <= KVM_ANCHOR_MAX_SEQ.  kvm_segment's sim_out then receives, per token, the
+                                    number of predecessors it would gather as a group's last state. */
     KVM_SETS_CONSERVED_ONLY = 1  /* eviction as in the heavy-hitter schemes of Section 2.2: only the conserved tokens
                                     (largest scores + most recent) stay, unchanged, in token order; pivot_rule,
                                     weight_rule, sim_threshold and sigma are ignored, out_len = n_recent + n_heavy,
@@ -106,6 +112,7 @@ enum kvm_set_rule {
 };
 
 #define KVM_MAX_SEQ 65536
+#define KVM_ANCHOR_MAX_SEQ 40960 /* longest sequence for KVM_SETS_ANCHOR (its walk lives in shared memory) */
 
 /* Device-side report, filled by kvm_segment / kvm_compress when given.  Zero it before the call. */
 typedef struct kvm_stats {

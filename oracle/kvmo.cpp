@@ -207,8 +207,10 @@ void kvmo_layer_ratio(int64_t U, int32_t S, double eps, const double* sim, doubl
 // run (nullable) [U,S] = for EVERY token i, the number of consecutive
 // predecessors whose similarity to k_i exceeds eps, ignoring conserved tokens
 // (the quantity the walk consults at its anchors).
+// run_in (nullable) [U,S]: run lengths decided elsewhere (e.g. in fp32 by the code under test); when given,
+// the walk consults them instead of evaluating cosines, so that only integer logic is left.
 void kvmo_boundaries_anchor(int64_t U, int32_t S, int32_t D, double eps, const float* K, const uint8_t* keep,
-                            uint8_t* b, int32_t* run) {
+                            uint8_t* b, int32_t* run, const int32_t* run_in) {
 #pragma omp parallel for schedule(static, 1)
     for (int64_t u = 0; u < U; ++u) {
         const float* Ku = K + (size_t)u * S * D;
@@ -231,8 +233,14 @@ void kvmo_boundaries_anchor(int64_t U, int32_t S, int32_t D, double eps, const f
         int32_t i = S - 1;
         while (i >= 0) {
             int32_t j = i - 1;
-            if (!kp[i])
-                while (j >= 0 && !kp[j] && cosine(i, j) > eps) --j;
+            if (!kp[i]) {
+                if (run_in) {
+                    int32_t left = run_in[(size_t)u * S + i];
+                    while (j >= 0 && !kp[j] && left > 0) { --j; --left; }
+                } else {
+                    while (j >= 0 && !kp[j] && cosine(i, j) > eps) --j;
+                }
+            }
             b[(size_t)u * S + j + 1] = 1;       // the group is tokens j+1 .. i
             i = j;
         }
@@ -439,7 +447,7 @@ void kvmo_compress(int32_t B, int32_t Hq, int32_t Hkv, int32_t S, int32_t D, dou
         }
         return;
     }
-    if (set_rule == 2) kvmo_boundaries_anchor(U, S, D, eps, K, keep, b, nullptr);   // no budget rule: cap must be S
+    if (set_rule == 2) kvmo_boundaries_anchor(U, S, D, eps, K, keep, b, nullptr, nullptr);   // no budget rule: cap must be S
     else kvmo_boundaries(U, S, cap, eps, enforce_budget, sim, keep, b, nullptr);
     kvmo_sets(U, S, cap, b, set_id, set_start, out_len);
     if (pivot_rule == 1) kvmo_pivots_last(U, cap, set_start, out_len, pivot);

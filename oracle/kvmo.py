@@ -111,8 +111,9 @@ def layer_ratio(sim: np.ndarray, eps: float) -> np.ndarray:
     return out
 
 
-def boundaries_anchor(K, keep_: np.ndarray, eps: float, want_run: bool = False):
-    """Anchor reading of the set identification (Section 3.2): flags [.., S], and the run length of every token."""
+def boundaries_anchor(K, keep_: np.ndarray, eps: float, want_run: bool = False, run_in=None):
+    """Anchor reading of the set identification (Section 3.2): flags [.., S], and the run length of every token.
+    With `run_in` the walk uses those run lengths instead of evaluating cosines."""
     K = _f32(K)
     keep_ = np.ascontiguousarray(keep_, dtype=np.uint8)
     S, D = K.shape[-2:]
@@ -120,7 +121,8 @@ def boundaries_anchor(K, keep_: np.ndarray, eps: float, want_run: bool = False):
     b = np.empty(K.shape[:-1], dtype=np.uint8)
     run = np.empty(K.shape[:-1], dtype=np.int32) if want_run else None
     lib().kvmo_boundaries_anchor(ctypes.c_int64(U), ctypes.c_int32(S), ctypes.c_int32(D), ctypes.c_double(eps),
-                                 _p(K), _p(keep_), _p(b), _p(run))
+                                 _p(K), _p(keep_), _p(b), _p(run),
+                                 _p(None if run_in is None else np.ascontiguousarray(run_in, dtype=np.int32)))
     return (b, run) if want_run else b
 
 

@@ -37,10 +37,11 @@ int derive(const kvm_params* p, Dims& d) {
     d.cap = d.enforce ? C : d.S;
     if (p->pivot_rule < KVM_PIVOT_MAX_SCORE || p->pivot_rule > KVM_PIVOT_KEY) return KVM_E_PARAM;
     if (p->weight_rule < KVM_WEIGHT_GAUSSIAN || p->weight_rule > KVM_WEIGHT_PIVOT_ONLY) return KVM_E_PARAM;
-    if (p->set_rule < KVM_SETS_ADJACENT || p->set_rule > KVM_SETS_CONSERVED_ONLY) return KVM_E_PARAM;
+    if (p->set_rule < KVM_SETS_ADJACENT || p->set_rule > KVM_SETS_ANCHOR) return KVM_E_PARAM;
+    if (p->set_rule == KVM_SETS_ANCHOR && (p->enforce_budget || p->seq > KVM_ANCHOR_MAX_SEQ)) return KVM_E_UNSUPPORTED;
     d.pivot_rule = p->pivot_rule; d.weight_rule = p->weight_rule; d.set_rule = p->set_rule;
     d.pivot_key = p->pivot_key;
-    if (p->set_rule == KVM_SETS_ADJACENT && p->weight_rule == KVM_WEIGHT_GAUSSIAN &&
+    if (p->set_rule != KVM_SETS_CONSERVED_ONLY && p->weight_rule == KVM_WEIGHT_GAUSSIAN &&
         (!(p->sigma > 0.f) || !isfinite(p->sigma)))
         return KVM_E_PARAM;
     if (d.set_rule == KVM_SETS_CONSERVED_ONLY) {
@@ -187,8 +188,11 @@ int kvm_segment(const kvm_params* p, const void* K, const float* scores, int32_t
     if ((rc = check_ws(d, ws, ws_bytes, w)) != KVM_OK) return rc;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     float* sim = sim_out ? sim_out : w.sim;
-    if (d.set_rule == KVM_SETS_ADJACENT || sim_out)
+    if (d.set_rule == KVM_SETS_ANCHOR) {
+        if (launch_anchor_runs(d, K, sim, st) != cudaSuccess) return KVM_E_CUDA;
+    } else if (d.set_rule == KVM_SETS_ADJACENT || sim_out) {
         if (launch_similarity(d, K, sim, st) != cudaSuccess) return KVM_E_CUDA;
+    }
     if (launch_segment(d, scores, sim, set_id, set_start, pivot, out_len, stats, st) != cudaSuccess)
         return KVM_E_CUDA;
     return KVM_OK;
@@ -290,6 +294,8 @@ int kvm_compress_with_lse(const kvm_params* p, const void* Q, const void* K, con
         return KVM_E_CUDA;
     if (want_sim && !sim_done)
         if (launch_similarity(d, K, w.sim, st) != cudaSuccess) return KVM_E_CUDA;
+    if (d.set_rule == KVM_SETS_ANCHOR)
+        if (launch_anchor_runs(d, K, w.sim, st) != cudaSuccess) return KVM_E_CUDA;
     if (launch_segment(d, scores, w.sim, w.set_id, w.set_start, out_pos, out_len, stats, st) != cudaSuccess)
         return KVM_E_CUDA;
     if (d.weight_rule == KVM_WEIGHT_PIVOT_ONLY)

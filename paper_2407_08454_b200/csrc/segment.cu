@@ -11,7 +11,9 @@
 //   5. segmented arg-max of the scores -> one pivot per set (or of the token
 //      index / a caller-supplied key, for the variants of Sections 4.2 and 5.3).
 // In eviction mode (Section 2.2) steps 2-5 are replaced by a compaction of the
-// conserved tokens.
+// conserved tokens.  Under the anchor reading of the set identification (Section
+// 3.2) steps 2-3 are replaced by a walk over per-token run lengths, done as
+// pointer jumping in shared memory.
 // Every tie is broken toward the lower token index, and every reduction has a
 // fixed order, so the integer outputs are reproducible bit for bit.
 #include <limits.h>
@@ -24,7 +26,7 @@ namespace {
 constexpr int NT = 1024;
 constexpr int NW = NT / 32;
 
-enum : uint8_t { F_KEEP = 1, F_HARD = 2, F_SOFT = 4, F_CUT = 8 };
+enum : uint8_t { F_KEEP = 1, F_HARD = 2, F_SOFT = 4, F_CUT = 8, F_ANCHOR = 16 };
 
 // Order-preserving map float -> uint32 (ascending).
 __device__ __forceinline__ uint32_t order_key(float f) {
@@ -66,6 +68,33 @@ __device__ __forceinline__ int block_exscan(int v, int& total, Shared& sh) {
     __syncthreads();
     total = sh.bcast[0];
     return sh.warp_i[w] + inc - v;
+}
+
+// Exclusive prefix maximum of one int per thread (identity -1).
+__device__ __forceinline__ int block_exscan_max(int v, Shared& sh) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    int inc = v;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, inc, off);
+        if (lane >= off) inc = max(inc, t);
+    }
+    __syncthreads();  // protect warp_i from a previous use
+    if (lane == 31) sh.warp_i[w] = inc;
+    __syncthreads();
+    if (w == 0) {
+        int x = sh.warp_i[lane];
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, x, off);
+            if (lane >= off) x = max(x, t);
+        }
+        const int ex = __shfl_up_sync(0xffffffffu, x, 1);
+        sh.warp_i[lane] = lane ? ex : -1;    // exclusive over warps
+    }
+    __syncthreads();
+    const int prev = __shfl_up_sync(0xffffffffu, inc, 1);
+    return max(sh.warp_i[w], lane ? prev : -1);
 }
 
 // Among the tokens j in [0, n) for which valid(j), find the k smallest keys (k >= 1,
@@ -133,7 +162,7 @@ __global__ void __launch_bounds__(NT) segment_unit_kernel(const float* __restric
                                                           int cap, int n_r, int n_h, float eps, int enforce,
                                                           int pivot_rule, const float* __restrict__ pivot_key,
                                                           int set_rule) {
-    extern __shared__ uint8_t flags[];  // [S]
+    extern __shared__ __align__(16) uint8_t flags[];  // [S] (+ jump arrays for the anchor reading)
     __shared__ Shared sh;
     const int u = blockIdx.x;
     const float* a = scores + (size_t)u * S;
@@ -200,6 +229,39 @@ __global__ void __launch_bounds__(NT) segment_unit_kernel(const float* __restric
         return;
     }
 
+    bool fire = false;
+    int tot_near = 0;
+    if (set_rule == KVM_SETS_ANCHOR) {
+        // ---- anchor reading (Section 3.2): token i, when it ends a group, takes with it the eff(i) tokens
+        // before it: its run length (c[] holds it) cut short by the nearest conserved token; conserved
+        // tokens take none.  The groups are the chain S-1 -> next(S-1) -> ... with next(i) = i - eff(i) - 1,
+        // found by pointer jumping: after round k every chain node within 2^k - 1 steps of S-1 is marked.
+        uint16_t* JA = reinterpret_cast<uint16_t*>(flags + ((S + 15) & ~15));     // next(i) + 1; 0 = chain ends
+        uint16_t* JB = JA + S;
+        int last_keep = -1;
+        for (int j = lo; j < hi; ++j) if (flags[j] & F_KEEP) last_keep = j;
+        int pk = block_exscan_max(last_keep, sh);            // nearest conserved token before this range
+        for (int j = lo; j < hi; ++j) {
+            const bool kept = (flags[j] & F_KEEP) != 0;
+            const int eff = kept ? 0 : min((int)c[j], j - 1 - pk);
+            JA[j] = (uint16_t)(j - eff);                      // next + 1 = j - eff - 1 + 1
+            if (kept) pk = j;
+        }
+        if (threadIdx.x == 0) flags[S - 1] |= F_ANCHOR;
+        __syncthreads();
+        unsigned* fw = reinterpret_cast<unsigned*>(flags);
+        for (int span = 1; span < S; span <<= 1) {
+            for (int j = lo; j < hi; ++j) {
+                const int nx = JA[j];
+                if ((flags[j] & F_ANCHOR) && nx) atomicOr(&fw[(nx - 1) >> 2], (unsigned)F_ANCHOR << (8 * ((nx - 1) & 3)));
+                JB[j] = nx ? JA[nx - 1] : (uint16_t)0;
+            }
+            __syncthreads();
+            uint16_t* t = JA; JA = JB; JB = t;
+        }
+        for (int j = lo; j < hi; ++j)
+            if (j == 0 || (flags[j - 1] & F_ANCHOR)) flags[j] |= F_CUT;   // own byte: neighbours read bit F_ANCHOR only
+    } else {
     // ---- 2. boundary flags
     int n_hard = 0, n_soft = 0, n_near = 0;
     for (int j = lo; j < hi; ++j) {
@@ -211,13 +273,13 @@ __global__ void __launch_bounds__(NT) segment_unit_kernel(const float* __restric
         else if (!(cj > eps)) { f |= F_SOFT | F_CUT; ++n_soft; }
         flags[j] = f;    // only bits other than F_KEEP change, so neighbours reading F_KEEP are safe
     }
-    int tot_hard, tot_soft, tot_near;
+    int tot_hard, tot_soft;
     block_exscan(n_hard, tot_hard, sh);
     block_exscan(n_soft, tot_soft, sh);
     block_exscan(n_near, tot_near, sh);
 
     // ---- 3. budget rule: keep only the (cap - hard) soft cuts with the smallest similarity
-    const bool fire = enforce && (tot_hard + tot_soft > cap);
+    fire = enforce && (tot_hard + tot_soft > cap);
     if (fire) {
         const int m = max(0, cap - tot_hard);
         uint32_t cut2 = 0;
@@ -243,6 +305,7 @@ __global__ void __launch_bounds__(NT) segment_unit_kernel(const float* __restric
             }
         }
     }
+    }   // neighbour reading
     __syncthreads();
 
     // ---- 4. scan of the cut flags -> set ids and starts
@@ -371,6 +434,12 @@ __global__ void __launch_bounds__(256) set_ratio_kernel(const float* __restrict_
 
 }  // namespace
 
+// Largest dynamic shared memory the segment kernel is ever launched with: the anchor reading at KVM_ANCHOR_MAX_SEQ.
+size_t segment_max_smem() {
+    const size_t a = (size_t)KVM_MAX_SEQ, b = (size_t)5 * KVM_ANCHOR_MAX_SEQ + 16;
+    return a > b ? a : b;
+}
+
 cudaError_t launch_set_ratio(const Dims& d, const float* sim, float* ratio, cudaStream_t st) {
     set_ratio_kernel<<<d.U, 256, 0, st>>>(sim, ratio, d.S, d.eps);
     return cudaGetLastError();
@@ -378,12 +447,14 @@ cudaError_t launch_set_ratio(const Dims& d, const float* sim, float* ratio, cuda
 
 cudaError_t launch_segment(const Dims& d, const float* scores, const float* sim, int32_t* set_id,
                            int32_t* set_start, int32_t* pivot, int32_t* out_len, kvm_stats* stats, cudaStream_t st) {
-    if (d.S > 40 * 1024) {   // more dynamic shared memory than the default limit: opt in (cheap, idempotent)
+    // flags [S] bytes; the anchor reading adds two uint16 jump arrays
+    const size_t smem = d.set_rule == KVM_SETS_ANCHOR ? (size_t)((d.S + 15) & ~15) + 4 * (size_t)d.S : (size_t)d.S;
+    if (smem > 40 * 1024) {   // more dynamic shared memory than the default limit: opt in (cheap, idempotent)
         cudaError_t e = cudaFuncSetAttribute(segment_unit_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             KVM_MAX_SEQ);
+                                             (int)segment_max_smem());
         if (e != cudaSuccess) return e;
     }
-    segment_unit_kernel<<<d.U, NT, (size_t)d.S, st>>>(scores, sim, set_id, set_start, pivot, out_len, stats, d.S,
+    segment_unit_kernel<<<d.U, NT, smem, st>>>(scores, sim, set_id, set_start, pivot, out_len, stats, d.S,
                                                      d.cap, d.n_r, d.n_h, d.eps, d.enforce, d.pivot_rule,
                                                      d.pivot_rule == KVM_PIVOT_KEY ? d.pivot_key : nullptr,
                                                      d.set_rule);

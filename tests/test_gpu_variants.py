@@ -96,3 +96,68 @@ def test_layer_ratio_and_per_layer_thresholds():
         g = run_gpu(Case(Q.cpu(), K.cpu(), V.cpu(), budget=cfg.budget, eps=eps))
         assert np.array_equal(o.out_len.cpu().numpy(), g.c_out_len)
     print("layer ratios", ratios, "compressed", r_lo, r_hi)
+
+
+@pytest.mark.parametrize("name,kw", SHAPES + [("C1", dict(seq=4096, n_q_heads=2, n_kv_heads=2, seed=23)),
+                                              ("C4", dict(seq=1500, n_q_heads=4, n_kv_heads=4, batch=1, seed=24))])
+def test_anchor_reading_of_the_set_identification(name, kw):
+    """Section 3.2's wording: similarity to the group's last state.  The run lengths are the only numbers floating
+    point decides: they must equal the checker's except where a pair lies within 1e-3 of the threshold, and given
+    the library's own run lengths and scores every integer output must equal the checker's integer-only walk."""
+    from oracle import kvmo
+    from parity import f32, kv_error, KV_TOL
+    case = _case(name, kw, set_rule=kvm.KVM_SETS_ANCHOR, enforce=False)
+    g = run_gpu(case)
+    B, Hq, S, D = case.Q.shape
+    U = B * case.K.shape[1]
+    cap, n_r, n_h = kvm.kvm_sizes(case.params())
+    assert cap == S
+    K = case.K.reshape(U, S, D)
+    eps = f32(case.eps)
+    g_run = g.sim.reshape(U, S)
+    assert (g_run == np.round(g_run)).all()
+    g_run = g_run.astype(np.int32)
+    keep = kvmo.keep(g.scores.reshape(U, S).astype(np.float64), n_r, n_h)
+    _, ref_run = kvmo.boundaries_anchor(K, keep, eps, want_run=True)
+    K64 = K.double().numpy()
+    differ = np.argwhere(g_run != ref_run)
+    for u, i in differ:                         # each disagreement needs a pair at the threshold
+        lo = max(0, i - max(g_run[u, i], ref_run[u, i]) - 1)
+        a = K64[u, i]
+        c = (K64[u, lo:i] @ a) / (np.linalg.norm(K64[u, lo:i], axis=1) * np.linalg.norm(a) + 1e-300)
+        assert np.abs(c - eps).min() < 1e-3, (u, i, g_run[u, i], ref_run[u, i])
+    assert len(differ) <= 0.01 * U * S
+    b = kvmo.boundaries_anchor(K, keep, eps, run_in=g_run)
+    set_id, st, ol = kvmo.sets(b, cap)
+    pv = kvmo.pivots(g.scores.reshape(U, S).astype(np.float64), st, ol)
+    assert np.array_equal(g.out_len.reshape(U), ol) and np.array_equal(g.set_id.reshape(U, S), set_id)
+    g_st, g_pv = g.set_start.reshape(U, cap + 1), g.pivot.reshape(U, cap)
+    rK, rV = kvmo.merge(K, case.V.reshape(U, S, D), st, pv, ol, f32(case.sigma), True)
+    for u in range(U):
+        n = ol[u]
+        assert np.array_equal(g_st[u, :n + 1], st[u, :n + 1]) and np.array_equal(g_pv[u, :n], pv[u, :n])
+        assert kv_error(g.K_out.reshape(U, cap, D)[u, :n], rK[u, :n]) <= KV_TOL
+        assert kv_error(g.V_out.reshape(U, cap, D)[u, :n], rV[u, :n]) <= KV_TOL
+        assert np.array_equal(g.c_out_pos.reshape(U, cap)[u, :n], pv[u, :n])
+        assert np.array_equal(g.c_K_out.reshape(U, cap, D)[u, :n], g.K_out.reshape(U, cap, D)[u, :n])
+    assert np.array_equal(g.c_out_len.reshape(U), ol)
+    print(name, kw, "sets", ol.tolist()[:4], "run disagreements", len(differ))
+
+
+def test_anchor_reading_limits():
+    with pytest.raises(kvm.KvmError) as e:      # needs the full capacity and a sequence that fits shared memory
+        kvm.kvm_sizes(kvm.make_params(1, 2, 2, 512, 64, torch.float32, set_rule=kvm.KVM_SETS_ANCHOR))
+    assert e.value.status == -7
+    with pytest.raises(kvm.KvmError) as e:
+        kvm.kvm_sizes(kvm.make_params(1, 2, 2, 40961, 64, torch.float32, set_rule=kvm.KVM_SETS_ANCHOR,
+                                      enforce_budget=0))
+    assert e.value.status == -7
+    # the longest accepted sequence runs (one unit), with the invariants of a partition
+    S = 40960
+    cfg = si.CONFIGS["C1"].scaled(seq=S, head_dim=64, n_q_heads=1, n_kv_heads=1, seed=25)
+    d = si.make_layer(cfg)
+    p = kvm.make_params(1, 1, 1, S, 64, torch.bfloat16, set_rule=kvm.KVM_SETS_ANCHOR, enforce_budget=0)
+    r = kvm.Compressor(p)(d["Q"].cuda(), d["K"].cuda(), d["V"].cuda())
+    n = int(r.out_len[0, 0])
+    pos = r.out_pos[0, 0, :n].cpu().numpy()
+    assert 1 <= n <= S and (np.diff(pos) > 0).all() and pos[-1] <= S - 1

@@ -203,6 +203,7 @@ def test_anchor_grouping_is_the_unique_partition_with_its_defining_properties():
                 continue
             assert all(_cos(x[0, hi], x[0, j]) > eps for j in range(lo, hi))
             assert lo == 0 or keep[0, lo - 1] or not (_cos(x[0, hi], x[0, lo - 1]) > eps)
+        np.testing.assert_array_equal(kvmo.boundaries_anchor(x, keep, eps, run_in=run), b)   # integer-only walk
         for i in range(S):                      # run lengths: brute force over every anchor candidate
             r = 0
             while i - 1 - r >= 0 and _cos(x[0, i], x[0, i - 1 - r]) > eps:
