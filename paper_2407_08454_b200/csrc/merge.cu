@@ -31,9 +31,6 @@ constexpr float LOG2E = 1.4426950408889634f;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-template <typename T> __device__ __forceinline__ float elem_to_f32(T v);
-template <> __device__ __forceinline__ float elem_to_f32<float>(float v) { return v; }
-template <> __device__ __forceinline__ float elem_to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
 template <typename T> __device__ __forceinline__ T f32_to_elem(float v);
 template <> __device__ __forceinline__ float f32_to_elem<float>(float v) { return v; }
 template <> __device__ __forceinline__ __nv_bfloat16 f32_to_elem<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }

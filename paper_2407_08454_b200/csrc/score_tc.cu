@@ -55,7 +55,6 @@ constexpr int SIM_RUN = 8;              // consecutive tokens per lane group and
 constexpr int NTHREADS = (NEPI_WARPS + 2 + NSIM_WARPS) * 32;
 constexpr long long WAIT_LIMIT_CLOCKS = 4000000000ll;   // ~2 s of SM clocks: a longer wait is reported, not endured
 constexpr float LOG2E = 1.4426950408889634f;
-constexpr float LN2 = 0.6931471805599453f;
 
 // ------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -215,11 +214,6 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
     float r;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
     return r;
-}
-__device__ __forceinline__ float hsum2(uint64_t p) {
-    float lo, hi;
-    unpack2(p, lo, hi);
-    return lo + hi;
 }
 __device__ __forceinline__ void named_bar(int id, int nthreads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
