@@ -51,6 +51,31 @@ template <> struct Vec<__nv_bfloat16> {
 
 __device__ __forceinline__ uint4 ldg16(const void* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
 
+// Programmatic dependent launch: a kernel launched with launch_dependent() may be scheduled while the kernel
+// before it on the stream is still draining; it must call grid_dependency_wait() before it touches anything that
+// kernel wrote (the wait returns once the earlier grid has completed and its writes are visible; it is a no-op for
+// a kernel launched the ordinary way).
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the kernel launched after this one (with launch_dependent) be scheduled once every block of this grid has
+// called it or exited; that kernel still waits for this grid's completion in its grid_dependency_wait().
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                             Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // Launchers (each enqueues on the stream and returns the launch status).
 cudaError_t launch_score_simt(const Dims& d, const void* Q, const void* K, const float* lse_in, float* lse_ws,
                               float* scores, cudaStream_t st);

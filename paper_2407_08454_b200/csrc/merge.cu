@@ -116,13 +116,16 @@ __global__ void __launch_bounds__(MERGE_NT) merge_tile_kernel(const T* __restric
         asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                      ::"r"(smem_u32(sV)), "l"(Vu + (size_t)tok0 * D), "r"(bytes), "r"(smem_u32(&bar)) : "memory");
     }
+    // The K and V rows are inputs; everything read from here on comes from the kernel before this one.
+    grid_dependency_wait();
     // per-token set data while the rows are in flight
     for (int j = threadIdx.x; j < ntok; j += MERGE_NT) {
-        const int sid = __ldg(set_id + (size_t)u * S + tok0 + j);
+        // written by the previous kernel while this block may already have been resident: read through L2
+        const int sid = __ldcg(set_id + (size_t)u * S + tok0 + j);
         s_sid[j] = sid;
-        s_piv[j] = __ldg(pivot + (size_t)u * cap + sid);
-        s_beg[j] = __ldg(st + sid);
-        s_end[j] = __ldg(st + sid + 1);
+        s_piv[j] = __ldcg(pivot + (size_t)u * cap + sid);
+        s_beg[j] = __ldcg(st + sid);
+        s_end[j] = __ldcg(st + sid + 1);
     }
     __syncthreads();                     // barrier initialised + metadata visible
     {
@@ -275,6 +278,7 @@ __global__ void __launch_bounds__(2 * D) merge_fixup_kernel(const int32_t* __res
                                                             T* __restrict__ K_out, T* __restrict__ V_out,
                                                             int32_t* __restrict__ out_size, Slots<D> slots, int S,
                                                             int cap, int Tn, int scale_v) {
+    grid_dependency_wait();     // the tile kernel's slots
     const int c = blockIdx.x + 1;                 // boundary between tiles c-1 and c
     const long long u = blockIdx.y;
     const int b = c * TOK;
@@ -354,15 +358,13 @@ cudaError_t launch_t(const Dims& d, const void* K, const void* V, const int32_t*
                                          (int)smem);
     if (e != cudaSuccess) return e;
     const float c = -LOG2E / (2.f * d.sigma * d.sigma);
-    merge_tile_kernel<T, D, TOK><<<dim3(Tn, d.U), MERGE_NT, smem, st>>>(
-        (const T*)K, (const T*)V, set_start, pivot, set_id, (T*)K_out, (T*)V_out, out_size, slots, d.S, d.cap, c,
-        d.scale_v, d.weight_rule == KVM_WEIGHT_AVERAGE ? 1 : 0);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    if (Tn > 1) {
-        merge_fixup_kernel<T, D, TOK><<<dim3(Tn - 1, d.U), 2 * D, 0, st>>>(set_start, set_id, (T*)K_out, (T*)V_out,
-                                                                          out_size, slots, d.S, d.cap, Tn, d.scale_v);
-        e = cudaGetLastError();
-    }
+    e = launch_dependent(merge_tile_kernel<T, D, TOK>, dim3(Tn, d.U), dim3(MERGE_NT), smem, st, (const T*)K,
+                         (const T*)V, set_start, pivot, set_id, (T*)K_out, (T*)V_out, out_size, slots, d.S, d.cap, c,
+                         d.scale_v, d.weight_rule == KVM_WEIGHT_AVERAGE ? 1 : 0);
+    if (e != cudaSuccess) return e;
+    if (Tn > 1)
+        e = launch_dependent(merge_fixup_kernel<T, D, TOK>, dim3(Tn - 1, d.U), dim3(2 * D), 0, st, set_start, set_id,
+                             (T*)K_out, (T*)V_out, out_size, slots, d.S, d.cap, Tn, d.scale_v);
     return e;
 }
 

@@ -321,6 +321,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     Shared& sh = *reinterpret_cast<Shared*>(sOnes + PTILE_BYTES);
     volatile int* abort_flag = &sh.abort_flag;
 
+    grid_dependency_wait();     // the column pass reads what the row pass (or the lse conversion) wrote
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = Hq / Hkv;
     const int T = (S + TILE - 1) / TILE;
@@ -685,9 +686,9 @@ cudaError_t launch_t(const Dims& d, const CUtensorMap& mq, const CUtensorMap& mk
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     const long long items = (long long)d.U * T;
     const int grid = (int)(items < sms ? items : sms);
-    score_tc_kernel<KCH><<<grid, NTHREADS, smem, st>>>(mq, mk, mp, nullptr, scores, stats, 2, d.B, d.Hq, d.Hkv, d.S,
-                                                      scale2, Ksim, sim_in_pass2 ? sim_out : nullptr);
-    return cudaGetLastError();
+    return launch_dependent(score_tc_kernel<KCH>, dim3(grid), dim3(NTHREADS), smem, st, mq, mk, mp,
+                            (__nv_bfloat16*)nullptr, scores, stats, 2, d.B, d.Hq, d.Hkv, d.S, scale2, Ksim,
+                            sim_in_pass2 ? sim_out : (float*)nullptr);
 }
 
 }  // namespace

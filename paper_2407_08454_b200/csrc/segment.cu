@@ -164,6 +164,10 @@ __global__ void __launch_bounds__(NT) segment_unit_kernel(const float* __restric
                                                           int set_rule) {
     extern __shared__ __align__(16) uint8_t flags[];  // [S] (+ jump arrays for the anchor reading)
     __shared__ Shared sh;
+    // One block per unit leaves most SMs idle: let the merge kernel's blocks move in now and stage their K and V
+    // tiles (inputs, never written) while this kernel runs; they wait for its results before reading any.
+    grid_launch_dependents();
+    grid_dependency_wait();     // scores and similarities come from the kernels before this one
     const int u = blockIdx.x;
     const float* a = scores + (size_t)u * S;
     const float* c = sim + (size_t)u * S;
@@ -454,11 +458,9 @@ cudaError_t launch_segment(const Dims& d, const float* scores, const float* sim,
                                              (int)segment_max_smem());
         if (e != cudaSuccess) return e;
     }
-    segment_unit_kernel<<<d.U, NT, smem, st>>>(scores, sim, set_id, set_start, pivot, out_len, stats, d.S,
-                                                     d.cap, d.n_r, d.n_h, d.eps, d.enforce, d.pivot_rule,
-                                                     d.pivot_rule == KVM_PIVOT_KEY ? d.pivot_key : nullptr,
-                                                     d.set_rule);
-    return cudaGetLastError();
+    return launch_dependent(segment_unit_kernel, dim3(d.U), dim3(NT), smem, st, scores, sim, set_id, set_start, pivot,
+                            out_len, stats, d.S, d.cap, d.n_r, d.n_h, d.eps, d.enforce, d.pivot_rule,
+                            d.pivot_rule == KVM_PIVOT_KEY ? d.pivot_key : (const float*)nullptr, d.set_rule);
 }
 
 }  // namespace kvm
