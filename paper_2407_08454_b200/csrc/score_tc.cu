@@ -676,8 +676,10 @@ cudaError_t launch_t(const Dims& d, const CUtensorMap& mq, const CUtensorMap& mk
     if (!lse_in) {
         const long long items = (long long)d.B * d.Hq * T;
         const int grid = (int)(items < sms ? items : sms);
-        score_tc_kernel<KCH><<<grid, NTHREADS, smem, st>>>(mq, mk, mp, side, nullptr, stats, 1, d.B, d.Hq, d.Hkv, d.S,
-                                                          scale2, Ksim, sim_out);
+        // (the kernel begins with the dependency wait, so it may be scheduled while whatever precedes it drains)
+        e = launch_dependent(score_tc_kernel<KCH>, dim3(grid), dim3(NTHREADS), smem, st, mq, mk, mp, side,
+                             (float*)nullptr, stats, 1, d.B, d.Hq, d.Hkv, d.S, scale2, Ksim, sim_out);
+        if (e != cudaSuccess) return e;
     } else {
         const long long rows = (long long)d.B * d.Hq * d.S;
         lse_split_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(lse_in, side, rows, -LOG2E / scale2);
