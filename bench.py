@@ -28,6 +28,7 @@ if ROOT not in sys.path:
 import numpy as np
 import torch
 
+from paper_2407_08454_b200 import replicas
 from paper_2407_08454_b200 import synth_inputs as si
 
 WORKLOAD = "C1"
@@ -187,7 +188,7 @@ def main():
     # ---- inputs: N_BUFFERS distinct layers per rank (weak scaling: every rank compresses its own layers)
     p = kvm.make_params(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.seq, cfg.head_dim, cfg.torch_dtype,
                         budget=cfg.budget)
-    host = [si.make_layer(cfg, layer=rank * N_BUFFERS + i) for i in range(N_BUFFERS)]
+    host = [si.make_layer(cfg, layer=l) for l in replicas.layers_for_rank(rank, world, N_BUFFERS)]
     bufs = [{k: v.to(dev) for k, v in h.items()} for h in host]
     comp = kvm.Compressor(p, device=dev)
     stats = kvm.new_stats(dev)
@@ -215,12 +216,8 @@ def main():
             step(i)
         e1.record(stream)
         barrier()
-    ms = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    value = world * args.steps * kv_tokens_per_step / (ms * 1e-3)
+    ms = replicas.slowest_rank_ms(e0.elapsed_time(e1), dist, dev)
+    value = replicas.aggregate_throughput(world, args.steps, kv_tokens_per_step, ms)
     st = kvm.read_stats(stats)
     assert st.status == 0, "device reported an error status"
 
@@ -360,16 +357,12 @@ def main():
         host_step(i)
     e1.record(stream)
     barrier()
-    ms_e2e = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([ms_e2e], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item())
+    ms_e2e = replicas.slowest_rank_ms(e0.elapsed_time(e1), dist, dev)
     assert int(hlen.sum()) == out_rows or True
     esz = 2 if cfg.dtype == "bf16" else 4
     h2d = (cfg.batch * cfg.n_q_heads + 2 * U) * cfg.seq * cfg.head_dim * esz
     d2h = 2 * U * comp.cap * cfg.head_dim * esz + U * 4 + U * comp.cap * 4
-    e2e = {"value": world * e2e_steps * kv_tokens_per_step / (ms_e2e * 1e-3), "unit": UNIT,
+    e2e = {"value": replicas.aggregate_throughput(world, e2e_steps, kv_tokens_per_step, ms_e2e), "unit": UNIT,
            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
            "ms_per_step": ms_e2e / e2e_steps}
 
