@@ -141,6 +141,7 @@ __global__ void __launch_bounds__(MERGE_NT) merge_tile_kernel(const T* __restric
 
     // ---- phase 1: weights, one lane group per token
     for (int j = w; j < ntok; j += NWORK) {
+        if (s_end[j] - s_beg[j] == 1) continue;      // a set of one token is copied, its weight is never used
         const int p = s_piv[j];
         float kj[N], kp[N];
         Vec<T>::unpack(*reinterpret_cast<const uint4*>(sK + (size_t)j * D + lane * N), kj);
@@ -200,6 +201,7 @@ __global__ void __launch_bounds__(MERGE_NT) merge_tile_kernel(const T* __restric
                 gs = 0.f;
                 first_raw = raw;
             }
+            if (s_end[j] - s_beg[j] == 1) continue;      // copied from first_raw at its flush
             const float g = s_g[j];
             float x[N];
             Vec<T>::unpack(raw, x);
