@@ -124,6 +124,7 @@ __global__ void __launch_bounds__(ATT_NT) attend_partial_kernel(const T* __restr
 template <int D>
 __global__ void __launch_bounds__(D) attend_combine_kernel(const float* __restrict__ part, float* __restrict__ out,
                                                            int nsplit) {
+    grid_dependency_wait();     // the partial states come from the kernel before this one
     const int bh = blockIdx.x;
     const float* p = part + (size_t)bh * nsplit * (D + 2);
     float M = -INFINITY;
@@ -143,6 +144,7 @@ template <int D>
 __global__ void __launch_bounds__(D) perturbation_kernel(const float* __restrict__ O, const float* __restrict__ Os,
                                                          float* __restrict__ err, float* __restrict__ ref) {
     __shared__ float se[D / 32], sr[D / 32];
+    grid_dependency_wait();     // both attention outputs come from the kernels before this one
     const int bh = blockIdx.x;
     const float a = O[(size_t)bh * D + threadIdx.x], c = Os[(size_t)bh * D + threadIdx.x];
     float e = (a - c) * (a - c), r = a * a;
@@ -170,8 +172,7 @@ cudaError_t launch_t(const Dims& d, const void* q, const void* K, const void* V,
         (const T*)q, (const T*)K, (const T*)V, len, part, rows, d.G, d.Hq, d.Hkv, d.scale * LOG2E);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    attend_combine_kernel<D><<<d.B * d.Hq, D, 0, st>>>(part, out, nsplit);
-    return cudaGetLastError();
+    return launch_dependent(attend_combine_kernel<D>, dim3(d.B * d.Hq), dim3(D), 0, st, (const float*)part, out, nsplit);
 }
 
 }  // namespace
@@ -192,9 +193,8 @@ cudaError_t launch_attend(const Dims& d, const void* q, const void* K, const voi
 
 cudaError_t launch_perturbation(const Dims& d, const float* O, const float* Os, float* err, float* ref,
                                 cudaStream_t st) {
-    if (d.D == 128) perturbation_kernel<128><<<d.B * d.Hq, 128, 0, st>>>(O, Os, err, ref);
-    else perturbation_kernel<64><<<d.B * d.Hq, 64, 0, st>>>(O, Os, err, ref);
-    return cudaGetLastError();
+    if (d.D == 128) return launch_dependent(perturbation_kernel<128>, dim3(d.B * d.Hq), dim3(128), 0, st, O, Os, err, ref);
+    return launch_dependent(perturbation_kernel<64>, dim3(d.B * d.Hq), dim3(64), 0, st, O, Os, err, ref);
 }
 
 }  // namespace kvm
