@@ -189,7 +189,8 @@ int kvm_segment(const kvm_params* p, const void* K, const float* scores, int32_t
     cudaStream_t st = (cudaStream_t)cuda_stream;
     float* sim = sim_out ? sim_out : w.sim;
     if (d.set_rule == KVM_SETS_ANCHOR) {
-        if (launch_anchor_runs(d, K, sim, st) != cudaSuccess) return KVM_E_CUDA;
+        // (the workspace's set-id region is free until the segment kernel writes it: scratch for the key norms)
+        if (launch_anchor_runs(d, K, sim, (float*)w.set_id, st) != cudaSuccess) return KVM_E_CUDA;
     } else if (d.set_rule == KVM_SETS_ADJACENT || sim_out) {
         if (launch_similarity(d, K, sim, st) != cudaSuccess) return KVM_E_CUDA;
     }
@@ -295,7 +296,7 @@ int kvm_compress_with_lse(const kvm_params* p, const void* Q, const void* K, con
     if (want_sim && !sim_done)
         if (launch_similarity(d, K, w.sim, st) != cudaSuccess) return KVM_E_CUDA;
     if (d.set_rule == KVM_SETS_ANCHOR)
-        if (launch_anchor_runs(d, K, w.sim, st) != cudaSuccess) return KVM_E_CUDA;
+        if (launch_anchor_runs(d, K, w.sim, (float*)w.set_id, st) != cudaSuccess) return KVM_E_CUDA;
     if (launch_segment(d, scores, w.sim, w.set_id, w.set_start, out_pos, out_len, stats, st) != cudaSuccess)
         return KVM_E_CUDA;
     if (d.weight_rule == KVM_WEIGHT_PIVOT_ONLY)

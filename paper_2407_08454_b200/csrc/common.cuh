@@ -86,7 +86,7 @@ cudaError_t launch_similarity(const Dims& d, const void* K, float* sim, cudaStre
 cudaError_t launch_segment(const Dims& d, const float* scores, const float* sim, int32_t* set_id,
                            int32_t* set_start, int32_t* pivot, int32_t* out_len, kvm_stats* stats, cudaStream_t st);
 size_t segment_max_smem();
-cudaError_t launch_anchor_runs(const Dims& d, const void* K, float* run_out, cudaStream_t st);
+cudaError_t launch_anchor_runs(const Dims& d, const void* K, float* run_out, float* inv_norm, cudaStream_t st);
 cudaError_t launch_set_ratio(const Dims& d, const float* sim, float* ratio, cudaStream_t st);
 size_t merge_scratch_floats(const Dims& d);
 cudaError_t launch_token_sets(const Dims& d, const int32_t* set_start, const int32_t* out_len, int32_t* set_id,
