@@ -258,6 +258,15 @@ def check_case(case: Case, g: Optional[GpuOut] = None, units: Optional[list] = N
             assert _near_tie_unit(case, ref_scores[i], ref_sim[i], {k: v for k, v in pure.items()}, i, cap, n_r,
                                   n_h), f"unit {sel[i]} differs from the fp64 chain without a near-tie"
             rep.units_near_tie += 1
+    # the device-side report of kvm_segment (all units only: it is a sum over the launch)
+    if units is None and case.set_rule == kvm.KVM_SETS_ADJACENT:
+        st_ = g.stats
+        assert st_.status == 0
+        assert (st_.min_out_len, st_.max_out_len, st_.sum_out_len) == (g_len.min(), g_len.max(), g_len.sum())
+        assert st_.units_budget_rule == int(np.count_nonzero(forced["fired"]))
+        near = np.abs(g_sim[:, 1:].astype(np.float32) - np.float32(case.eps)) < np.float32(1e-3)
+        assert st_.near_threshold == int(near.sum())
+
     # kvm_compress must agree with the step-by-step calls bit for bit
     assert np.array_equal(unit_view(g.c_out_len, ()), g_len)
     c_pos, c_K, c_V = unit_view(g.c_out_pos, (cap,)), unit_view(g.c_K_out, (cap, D)), unit_view(g.c_V_out, (cap, D))
