@@ -15,7 +15,8 @@
 // Parity pins (tests/test_oracle_*.py): every function below is pinned by
 // closed forms, invariants or brute force.  Parity unpinned BY THE PAPER (no
 // printed example; pinned only by brute force, monotonicity and invariants):
-// the budget rule in kvmo_boundaries.
+// the budget rule in kvmo_boundaries; the per-set bandwidth of kvmo_merge's
+// weight_rule 3 (a reading of Eq. 4, which is circular as printed).
 #include <cmath>
 #include <cstdint>
 #include <cstring>
@@ -297,6 +298,10 @@ void kvmo_pivots_last(int64_t U, int32_t cap, const int32_t* set_start, const in
 // weight_rule 0 is the paper's method.  1 = average-weighted merging (Section
 // 4.2's baseline): g_j = 1, so w_j = 1/|set|.  2 = the sigma -> 0 limit named
 // after Eq. 5: nothing but the pivot survives, g_j = [j == p].
+// 3 = a bandwidth per merging set (PARITY UNPINNED: Eq. 4 defines sigma through
+// the weights that depend on it; this is one non-circular reading, not the
+// paper's statement): sigma_s^2 = mean_{j in set} |k_p - k_j|^2 / 2, i.e.
+// g_j = exp(-|k_p - k_j|^2 / mean_t |k_p - k_t|^2), and g_j = 1 when that mean is 0.
 // K_out, V_out [U,cap,D] fp64 (rows >= out_len untouched); weights (nullable) [U,S].
 void kvmo_merge(int64_t U, int32_t S, int32_t D, int32_t cap, double sigma, int32_t scale_v, int32_t weight_rule,
                 const float* K, const float* V, const int32_t* set_start, const int32_t* pivot,
@@ -310,7 +315,18 @@ void kvmo_merge(int64_t U, int32_t S, int32_t D, int32_t cap, double sigma, int3
         for (int32_t s = 0; s < out_len[u]; ++s) {
             const int32_t lo = st[s], hi = st[s + 1], p = pivot[(size_t)u * cap + s];
             const float* kp = Ku + (size_t)p * D;
-            double gsum = 0.0;
+            double gsum = 0.0, two_sigma2 = 2.0 * sigma * sigma;
+            if (weight_rule == 3) {
+                double total = 0.0;
+                for (int32_t j = lo; j < hi; ++j) {
+                    const float* kj = Ku + (size_t)j * D;
+                    for (int32_t t = 0; t < D; ++t) {
+                        const double df = (double)kp[t] - (double)kj[t];
+                        total += df * df;
+                    }
+                }
+                two_sigma2 = total / (double)(hi - lo);      // 2 sigma_s^2 = mean squared distance to the pivot
+            }
             for (int32_t j = lo; j < hi; ++j) {
                 const float* kj = Ku + (size_t)j * D;
                 double d2 = 0.0;
@@ -320,7 +336,8 @@ void kvmo_merge(int64_t U, int32_t S, int32_t D, int32_t cap, double sigma, int3
                 }
                 if (weight_rule == 1) g[j] = 1.0;
                 else if (weight_rule == 2) g[j] = (j == p) ? 1.0 : 0.0;
-                else g[j] = std::exp(-d2 / (2.0 * sigma * sigma));
+                else if (weight_rule == 3 && !(two_sigma2 > 0.0)) g[j] = 1.0;
+                else g[j] = std::exp(-d2 / two_sigma2);
                 gsum += g[j];
             }
             double* ko = K_out + ((size_t)u * cap + s) * D;

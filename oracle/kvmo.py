@@ -178,7 +178,7 @@ def evict(keep_: np.ndarray, K, V, cap: int):
 
 
 PIVOT_MAX_SCORE, PIVOT_LAST, PIVOT_KEY = 0, 1, 2
-WEIGHT_GAUSSIAN, WEIGHT_AVERAGE, WEIGHT_PIVOT_ONLY = 0, 1, 2
+WEIGHT_GAUSSIAN, WEIGHT_AVERAGE, WEIGHT_PIVOT_ONLY, WEIGHT_SET_SIGMA = 0, 1, 2, 3
 SETS_ADJACENT, SETS_CONSERVED_ONLY, SETS_ANCHOR = 0, 1, 2
 
 

@@ -252,3 +252,51 @@ def test_compress_with_anchor_sets_equals_its_steps():
     np.testing.assert_array_equal(kvmo.pivots(r.scores, st, ol), r.pivot)
     base = kvmo.compress(d["Q"], d["K"], d["V"], 0.50, 0.17, 0.12, enforce_budget=False)
     assert (r.out_len >= base.out_len).all()        # similarity to the anchor is the stricter requirement here
+
+
+# ---------------------------------------------------------------- bandwidth per merging set (a reading of Eq. 4)
+def test_set_sigma_rule_is_the_fixed_rule_at_the_set_own_bandwidth():
+    K, V = _rand((1, 60, 6), 30), _rand((1, 60, 6), 31)
+    set_id, st, ol = _random_partition(60, 1, 32)
+    pv = kvmo.pivots(_rand((1, 60), 33), st, ol)
+    Ko, Vo, w = kvmo.merge(K, V, st, pv, ol, sigma=123.0, scale_v=False, want_weights=True,
+                           weight_rule=kvmo.WEIGHT_SET_SIGMA)          # sigma is ignored
+    K64 = K.astype(np.float64)
+    for s in range(ol[0]):
+        lo, hi, p = st[0, s], st[0, s + 1], pv[0, s]
+        d2 = ((K64[0, lo:hi] - K64[0, p]) ** 2).sum(-1)
+        if hi - lo == 1:
+            np.testing.assert_array_equal(Ko[0, s], K64[0, lo])
+            continue
+        sigma_s = np.sqrt(d2.mean() / 2.0)
+        one = (np.array([[0, hi - lo]], np.int32), np.array([[p - lo]], np.int32), np.array([1], np.int32))
+        Kf, Vf, wf = kvmo.merge(K[:, lo:hi], V[:, lo:hi], *one, sigma=sigma_s, scale_v=False, want_weights=True)
+        np.testing.assert_allclose(Ko[0, s], Kf[0, 0], rtol=1e-12, atol=1e-14)
+        np.testing.assert_allclose(w[0, lo:hi], wf[0], rtol=1e-12)
+        np.testing.assert_allclose(np.log(w[0, lo:hi] / w[0, p]), -d2 / d2.mean(), rtol=1e-10, atol=1e-12)
+
+
+def test_set_sigma_rule_closed_forms_and_scale_invariance():
+    # two tokens: mean squared distance = d^2 / 2, so the other token's kernel value is exp(-2) whatever d is
+    for d in (0.1, 3.0, 50.0):
+        K = np.array([[[0.0, 0.0], [d, 0.0]]], np.float32)
+        V = np.array([[[1.0, 0.0], [0.0, 1.0]]], np.float32)
+        st, pv, ol = np.array([[0, 2]], np.int32), np.array([[0]], np.int32), np.array([1], np.int32)
+        _, Vo, w = kvmo.merge(K, V, st, pv, ol, sigma=5.0, scale_v=False, want_weights=True,
+                              weight_rule=kvmo.WEIGHT_SET_SIGMA)
+        g = np.exp(-2.0)
+        np.testing.assert_allclose(w[0], [1 / (1 + g), g / (1 + g)], rtol=1e-14)
+    # identical keys: every kernel value is 1 -> uniform weights
+    K = np.repeat(_rand((1, 1, 4), 34), 5, axis=1)
+    st, pv, ol = np.array([[0, 5]], np.int32), np.array([[2]], np.int32), np.array([1], np.int32)
+    _, _, w = kvmo.merge(K, _rand((1, 5, 4), 35), st, pv, ol, 5.0, want_weights=True, weight_rule=kvmo.WEIGHT_SET_SIGMA)
+    np.testing.assert_allclose(w[0], 0.2, rtol=1e-15)
+    # rescaling all keys leaves the weights unchanged (the fixed-sigma rule does not have this property)
+    K, V = _rand((1, 9, 4), 36), _rand((1, 9, 4), 37)
+    st, pv, ol = np.array([[0, 9]], np.int32), np.array([[4]], np.int32), np.array([1], np.int32)
+    w1 = kvmo.merge(K, V, st, pv, ol, 5.0, want_weights=True, weight_rule=kvmo.WEIGHT_SET_SIGMA)[2]
+    w2 = kvmo.merge(4 * K, V, st, pv, ol, 5.0, want_weights=True, weight_rule=kvmo.WEIGHT_SET_SIGMA)[2]
+    np.testing.assert_allclose(w2, w1, rtol=1e-12)
+    f1 = kvmo.merge(K, V, st, pv, ol, 5.0, want_weights=True)[2]
+    f2 = kvmo.merge(4 * K, V, st, pv, ol, 5.0, want_weights=True)[2]
+    assert np.abs(f2 - f1).max() > 1e-3
