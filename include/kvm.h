@@ -92,8 +92,12 @@ enum kvm_pivot_rule {
 enum kvm_weight_rule {
     KVM_WEIGHT_GAUSSIAN = 0,  /* Eq. 4, Eq. 5 with the fixed sigma */
     KVM_WEIGHT_AVERAGE = 1,   /* every state 1/|set| (average-weighted merging, Section 4.2); sigma is ignored */
-    KVM_WEIGHT_PIVOT_ONLY = 2 /* the sigma -> 0 limit noted after Eq. 5: the pivot's own K and V rows, nothing
-                                 merged in (V still times the set size when scale_v_by_set_size) */
+    KVM_WEIGHT_PIVOT_ONLY = 2, /* the sigma -> 0 limit noted after Eq. 5: the pivot's own K and V rows, nothing
+                                  merged in (V still times the set size when scale_v_by_set_size) */
+    KVM_WEIGHT_SET_SIGMA = 3   /* a bandwidth per merging set.  Eq. 4 defines sigma through the weights that depend
+                                  on it; this rule is one non-circular reading, not the paper's statement:
+                                  2 sigma_s^2 = mean over the set of |k_p - k_j|^2, so g_j = exp(-|k_p - k_j|^2 / mean)
+                                  (every g_j = 1 when the mean is 0).  sigma is ignored. */
 };
 /* Which states reach the output. */
 enum kvm_set_rule {

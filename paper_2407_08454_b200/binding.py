@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_PKG, "libkvm.so")
 KVM_BF16, KVM_F32 = 0, 1
 KVM_OK = 0
 KVM_PIVOT_MAX_SCORE, KVM_PIVOT_LAST, KVM_PIVOT_KEY = 0, 1, 2
-KVM_WEIGHT_GAUSSIAN, KVM_WEIGHT_AVERAGE, KVM_WEIGHT_PIVOT_ONLY = 0, 1, 2
+KVM_WEIGHT_GAUSSIAN, KVM_WEIGHT_AVERAGE, KVM_WEIGHT_PIVOT_ONLY, KVM_WEIGHT_SET_SIGMA = 0, 1, 2, 3
 KVM_SETS_ADJACENT, KVM_SETS_CONSERVED_ONLY, KVM_SETS_ANCHOR = 0, 1, 2
 EXPORTS = (
     "kvm_sizes", "kvm_workspace_bytes", "kvm_score", "kvm_segment", "kvm_merge_compact", "kvm_compress",

@@ -36,7 +36,7 @@ int derive(const kvm_params* p, Dims& d) {
     d.enforce = p->enforce_budget ? 1 : 0;
     d.cap = d.enforce ? C : d.S;
     if (p->pivot_rule < KVM_PIVOT_MAX_SCORE || p->pivot_rule > KVM_PIVOT_KEY) return KVM_E_PARAM;
-    if (p->weight_rule < KVM_WEIGHT_GAUSSIAN || p->weight_rule > KVM_WEIGHT_PIVOT_ONLY) return KVM_E_PARAM;
+    if (p->weight_rule < KVM_WEIGHT_GAUSSIAN || p->weight_rule > KVM_WEIGHT_SET_SIGMA) return KVM_E_PARAM;
     if (p->set_rule < KVM_SETS_ADJACENT || p->set_rule > KVM_SETS_ANCHOR) return KVM_E_PARAM;
     if (p->set_rule == KVM_SETS_ANCHOR && (p->enforce_budget || p->seq > KVM_ANCHOR_MAX_SEQ)) return KVM_E_UNSUPPORTED;
     d.pivot_rule = p->pivot_rule; d.weight_rule = p->weight_rule; d.set_rule = p->set_rule;
@@ -263,7 +263,9 @@ int kvm_merge_compact(const kvm_params* p, const void* K, const void* V, const i
                    ? KVM_OK
                    : KVM_E_CUDA;
     if (launch_token_sets(d, set_start, out_len, w.set_id, st) != cudaSuccess) return KVM_E_CUDA;
-    return launch_merge(d, K, V, set_start, pivot, w.set_id, K_out, V_out, out_size, w.merge_part, st) == cudaSuccess
+    // (the similarity region of the workspace is free here: scratch for the per-set bandwidths)
+    return launch_merge(d, K, V, set_start, pivot, w.set_id, out_len, K_out, V_out, out_size, w.merge_part, w.sim, st) ==
+                   cudaSuccess
                ? KVM_OK
                : KVM_E_CUDA;
 }
@@ -303,7 +305,8 @@ int kvm_compress_with_lse(const kvm_params* p, const void* Q, const void* K, con
         return launch_gather(d, K, V, w.set_start, out_pos, out_len, K_out, V_out, nullptr, st) == cudaSuccess
                    ? KVM_OK
                    : KVM_E_CUDA;
-    if (launch_merge(d, K, V, w.set_start, out_pos, w.set_id, K_out, V_out, nullptr, w.merge_part, st) != cudaSuccess)
+    if (launch_merge(d, K, V, w.set_start, out_pos, w.set_id, out_len, K_out, V_out, nullptr, w.merge_part, w.sim, st) !=
+        cudaSuccess)
         return KVM_E_CUDA;
     return KVM_OK;
 }

@@ -81,7 +81,7 @@ __global__ void __launch_bounds__(MERGE_NT) merge_tile_kernel(const T* __restric
                                                               T* __restrict__ K_out, T* __restrict__ V_out,
                                                               int32_t* __restrict__ out_size, Slots<D> slots, int S,
                                                               int cap, float neg_inv_2s2_log2e, int scale_v,
-                                                              int average) {
+                                                              int average, const float* __restrict__ set_coef) {
     using Gm = MergeGeom<T, D>;
     constexpr int N = Gm::N, LPR = Gm::LPR, NWORK = Gm::NWORK, NCH = Gm::NCH;
     constexpr int CHL = TOK / NCH;                    // tokens per chunk
@@ -94,6 +94,7 @@ __global__ void __launch_bounds__(MERGE_NT) merge_tile_kernel(const T* __restric
     __shared__ __align__(8) uint64_t bar;
     __shared__ int s_sid[TOK], s_piv[TOK], s_beg[TOK], s_end[TOK];
     __shared__ float s_g[TOK];
+    __shared__ float s_coef[TOK];       // squared distance -> exponent of 2, per token (fixed sigma or the set's own)
     __shared__ float s_gpart[NCH][2];
 
     const int tile = blockIdx.x, Tn = gridDim.x;
@@ -126,6 +127,7 @@ __global__ void __launch_bounds__(MERGE_NT) merge_tile_kernel(const T* __restric
         s_piv[j] = __ldcg(pivot + (size_t)u * cap + sid);
         s_beg[j] = __ldcg(st + sid);
         s_end[j] = __ldcg(st + sid + 1);
+        s_coef[j] = set_coef ? __ldcg(set_coef + (size_t)u * cap + sid) : neg_inv_2s2_log2e;
     }
     __syncthreads();                     // barrier initialised + metadata visible
     {
@@ -154,7 +156,7 @@ __global__ void __launch_bounds__(MERGE_NT) merge_tile_kernel(const T* __restric
         for (int e = 0; e < N; ++e) { const float a = kp[e] - kj[e]; d2 = fmaf(a, a, d2); }
 #pragma unroll
         for (int off = 1; off < LPR; off <<= 1) d2 += __shfl_xor_sync(gmask, d2, off);
-        if (lane == 0) s_g[j] = average ? 1.f : exp2f(d2 * neg_inv_2s2_log2e);
+        if (lane == 0) s_g[j] = average ? 1.f : exp2f(d2 * s_coef[j]);
     }
     __syncthreads();
 
@@ -305,6 +307,38 @@ __global__ void __launch_bounds__(2 * D) merge_fixup_kernel(const int32_t* __res
     if (out_size && threadIdx.x == 0) out_size[(size_t)u * cap + sid] = n;
 }
 
+// Bandwidth per merging set (one non-circular reading of Eq. 4): 2 sigma_s^2 = mean over the set of
+// |k_p - k_j|^2.  Writes, per set, the factor that turns a squared distance into the exponent of 2:
+// coef = -log2(e) / mean, or 0 (every weight 1) when the mean is 0.  One lane group per set.
+template <typename T, int D>
+__global__ void __launch_bounds__(256) set_bandwidth_kernel(const T* __restrict__ K,
+                                                            const int32_t* __restrict__ set_start,
+                                                            const int32_t* __restrict__ pivot,
+                                                            const int32_t* __restrict__ out_len,
+                                                            float* __restrict__ coef, int S, int cap) {
+    constexpr int N = Vec<T>::N, LPR = D / N, SETS = 256 / LPR;
+    grid_dependency_wait();
+    const long long u = blockIdx.y;
+    const int s = blockIdx.x * SETS + threadIdx.x / LPR, lane = threadIdx.x % LPR;
+    if (s >= min(__ldcg(out_len + u), cap)) return;       // whole groups leave together
+    const unsigned gmask = (LPR == 32) ? 0xffffffffu : (((1u << LPR) - 1u) << ((threadIdx.x % 32) / LPR * LPR));
+    const int32_t* st = set_start + (size_t)u * (cap + 1);
+    const int lo = __ldcg(st + s), hi = __ldcg(st + s + 1), p = __ldcg(pivot + (size_t)u * cap + s);
+    const T* Ku = K + (size_t)u * S * D;
+    float kp[N];
+    Vec<T>::unpack(ldg16(Ku + (size_t)p * D + lane * N), kp);
+    float tot = 0.f;
+    for (int j = lo; j < hi; ++j) {
+        float kj[N];
+        Vec<T>::unpack(ldg16(Ku + (size_t)j * D + lane * N), kj);
+#pragma unroll
+        for (int e = 0; e < N; ++e) { const float a = kp[e] - kj[e]; tot = fmaf(a, a, tot); }
+    }
+#pragma unroll
+    for (int off = 1; off < LPR; off <<= 1) tot += __shfl_xor_sync(gmask, tot, off);
+    if (lane == 0) coef[(size_t)u * cap + s] = tot > 0.f ? -LOG2E * (float)(hi - lo) / tot : 0.f;
+}
+
 // Output rows that are a single input state: row s = K[pivot[s]], V[pivot[s]] (V times the set size when
 // asked and the sets are real ones).  One lane group per (row, tensor), 16-byte copies.
 template <typename T, int D>
@@ -349,8 +383,8 @@ cudaError_t launch_gather_t(const Dims& d, const void* K, const void* V, const i
 
 template <typename T, int D, int TOK>
 cudaError_t launch_t(const Dims& d, const void* K, const void* V, const int32_t* set_start, const int32_t* pivot,
-                     const int32_t* set_id, void* K_out, void* V_out, int32_t* out_size, float* scratch,
-                     cudaStream_t st) {
+                     const int32_t* set_id, const int32_t* out_len, void* K_out, void* V_out, int32_t* out_size,
+                     float* scratch, float* set_coef, cudaStream_t st) {
     const int Tn = (d.S + TOK - 1) / TOK;
     Slots<D> slots;
     slots.sums = scratch;
@@ -360,9 +394,17 @@ cudaError_t launch_t(const Dims& d, const void* K, const void* V, const int32_t*
                                          (int)smem);
     if (e != cudaSuccess) return e;
     const float c = -LOG2E / (2.f * d.sigma * d.sigma);
+    const bool per_set = d.weight_rule == KVM_WEIGHT_SET_SIGMA;
+    if (per_set) {
+        constexpr int SETS = 256 / (D / Vec<T>::N);
+        e = launch_dependent(set_bandwidth_kernel<T, D>, dim3((d.cap + SETS - 1) / SETS, d.U), dim3(256), 0, st,
+                             (const T*)K, set_start, pivot, out_len, set_coef, d.S, d.cap);
+        if (e != cudaSuccess) return e;
+    }
     e = launch_dependent(merge_tile_kernel<T, D, TOK>, dim3(Tn, d.U), dim3(MERGE_NT), smem, st, (const T*)K,
                          (const T*)V, set_start, pivot, set_id, (T*)K_out, (T*)V_out, out_size, slots, d.S, d.cap, c,
-                         d.scale_v, d.weight_rule == KVM_WEIGHT_AVERAGE ? 1 : 0);
+                         d.scale_v, d.weight_rule == KVM_WEIGHT_AVERAGE ? 1 : 0,
+                         per_set ? (const float*)set_coef : (const float*)nullptr);
     if (e != cudaSuccess) return e;
     if (Tn > 1)
         e = launch_dependent(merge_fixup_kernel<T, D, TOK>, dim3(Tn - 1, d.U), dim3(2 * D), 0, st, set_start, set_id,
@@ -402,18 +444,20 @@ cudaError_t launch_gather(const Dims& d, const void* K, const void* V, const int
                       : launch_gather_t<float, 64>(d, K, V, set_start, pivot, out_len, K_out, V_out, out_size, st);
 }
 
+// set_coef: [U, cap] fp32 of scratch, used only by the per-set bandwidth rule; out_len: device [U].
 cudaError_t launch_merge(const Dims& d, const void* K, const void* V, const int32_t* set_start,
-                         const int32_t* pivot, const int32_t* set_id, void* K_out, void* V_out, int32_t* out_size,
-                         float* scratch, cudaStream_t st) {
+                         const int32_t* pivot, const int32_t* set_id, const int32_t* out_len, void* K_out,
+                         void* V_out, int32_t* out_size, float* scratch, float* set_coef, cudaStream_t st) {
     if (d.dtype == KVM_BF16) {
-        return d.D == 128 ? launch_t<__nv_bfloat16, 128, KVM_MERGE_TOK_BF16>(d, K, V, set_start, pivot, set_id, K_out, V_out,
-                                                              out_size, scratch, st)
-                          : launch_t<__nv_bfloat16, 64, KVM_MERGE_TOK_BF16>(d, K, V, set_start, pivot, set_id, K_out, V_out,
-                                                             out_size, scratch, st);
+        return d.D == 128 ? launch_t<__nv_bfloat16, 128, KVM_MERGE_TOK_BF16>(d, K, V, set_start, pivot, set_id, out_len,
+                                                                          K_out, V_out, out_size, scratch, set_coef, st)
+                          : launch_t<__nv_bfloat16, 64, KVM_MERGE_TOK_BF16>(d, K, V, set_start, pivot, set_id, out_len,
+                                                                         K_out, V_out, out_size, scratch, set_coef, st);
     }
-    return d.D == 128
-               ? launch_t<float, 128, 64>(d, K, V, set_start, pivot, set_id, K_out, V_out, out_size, scratch, st)
-               : launch_t<float, 64, 64>(d, K, V, set_start, pivot, set_id, K_out, V_out, out_size, scratch, st);
+    return d.D == 128 ? launch_t<float, 128, 64>(d, K, V, set_start, pivot, set_id, out_len, K_out, V_out, out_size,
+                                                 scratch, set_coef, st)
+                      : launch_t<float, 64, 64>(d, K, V, set_start, pivot, set_id, out_len, K_out, V_out, out_size,
+                                                scratch, set_coef, st);
 }
 
 }  // namespace kvm

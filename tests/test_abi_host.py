@@ -70,7 +70,7 @@ def test_variant_parameter_checks(lib):
     with pytest.raises(kvm.KvmError) as e:
         kvm.kvm_sizes(p)
     assert e.value.status == -1
-    for bad in (dict(pivot_rule=3), dict(weight_rule=-1), dict(set_rule=3)):
+    for bad in (dict(pivot_rule=3), dict(weight_rule=4), dict(set_rule=3)):
         with pytest.raises(kvm.KvmError) as e:
             kvm.kvm_sizes(kvm.make_params(1, 2, 2, 256, 64, kvm.KVM_F32, **bad))
         assert e.value.status == -4

@@ -161,3 +161,17 @@ def test_anchor_reading_limits():
     n = int(r.out_len[0, 0])
     pos = r.out_pos[0, 0, :n].cpu().numpy()
     assert 1 <= n <= S and (np.diff(pos) > 0).all() and pos[-1] <= S - 1
+
+
+@pytest.mark.parametrize("name,kw", SHAPES)
+def test_bandwidth_per_merging_set(name, kw):
+    # one non-circular reading of Eq. 4 (parity unpinned by the paper): 2 sigma^2 = the set's mean squared
+    # distance to its pivot; the sets and pivots are those of the method
+    for scale_v in (False, True):
+        case = _case(name, kw, weight_rule=kvm.KVM_WEIGHT_SET_SIGMA, scale_v=scale_v, sigma=0.0)
+        g = run_gpu(case)
+        rep = check_case(case, g)
+        print(name, kw, scale_v, rep)
+    base = run_gpu(_case(name, kw))
+    assert np.array_equal(g.set_start, base.set_start) and np.array_equal(g.pivot, base.pivot)
+    assert not np.array_equal(g.K_out, base.K_out)
