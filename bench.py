@@ -308,6 +308,7 @@ def main():
                                                             weight_rule=kvm.KVM_WEIGHT_AVERAGE)),
         "compress_keyed_pivot_ms": t_compress(params(pivot_rule=kvm.KVM_PIVOT_KEY, pivot_key=key)),
         "compress_pivot_only_ms": t_compress(params(weight_rule=kvm.KVM_WEIGHT_PIVOT_ONLY)),
+        "compress_set_sigma_ms": t_compress(params(weight_rule=kvm.KVM_WEIGHT_SET_SIGMA)),
         "compress_eviction_ms": t_compress(params(set_rule=kvm.KVM_SETS_CONSERVED_ONLY, recent_ratio=0.17,
                                                   heavy_ratio=cfg.budget - 0.17)),
     }
