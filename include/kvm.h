@@ -69,7 +69,7 @@ typedef struct kvm_params {
     float recent_ratio;          /* share of S conserved as most recent tokens; < 0: preset 0.17 (budget >= 0.425) else 0.08 */
     float heavy_ratio;           /* share of S conserved for largest scores;    < 0: preset 0.12 (budget >= 0.425) else 0.02 */
     float sim_threshold;         /* epsilon of Algorithm 1; neighbours group when similarity > epsilon (strict); paper: 0.75 */
-    float sigma;                 /* Gaussian bandwidth of Eq. 4, > 0; the paper's best fixed value is 5 */
+    float sigma;                 /* Gaussian bandwidth of Eq. 4, > 0 (only KVM_WEIGHT_GAUSSIAN reads it); the paper's best fixed value is 5 */
     float softmax_scale;         /* <= 0: 1/sqrt(head_dim) as in Eq. 1 */
     int32_t causal;              /* must be 1 */
     int32_t scale_v_by_set_size; /* 1: value weights are multiplied by the set size (text after Eq. 5); 0: plain weighted mean */
@@ -102,17 +102,17 @@ enum kvm_weight_rule {
 /* Which states reach the output. */
 enum kvm_set_rule {
     KVM_SETS_ADJACENT = 0,       /* Algorithm 1: every token belongs to a merging set */
-    KVM_SETS_ANCHOR = 2,         /* the set identification as Section 3.2 words it: walking from the last token, a
+    KVM_SETS_CONSERVED_ONLY = 1, /* eviction as in the heavy-hitter schemes of Section 2.2: only the conserved tokens
+                                    (largest scores + most recent) stay, unchanged, in token order; pivot_rule,
+                                    weight_rule, sim_threshold and sigma are ignored, out_len = n_recent + n_heavy,
+                                    which must fit the capacity; set_id is -1 for dropped tokens and
+                                    set_start[s] = pivot[s] = the s-th kept token */
+    KVM_SETS_ANCHOR = 2          /* the set identification as Section 3.2 words it: walking from the last token, a
                                     state gathers the consecutive states before it whose similarity TO IT exceeds
                                     sim_threshold (Algorithm 1's listing compares neighbours instead).  Conserved
                                     tokens stand alone.  No budget rule: enforce_budget must be 0 (capacity S), and
                                     seq <= KVM_ANCHOR_MAX_SEQ.  kvm_segment's sim_out then receives, per token, the
                                     number of predecessors it would gather as a group's last state. */
-    KVM_SETS_CONSERVED_ONLY = 1  /* eviction as in the heavy-hitter schemes of Section 2.2: only the conserved tokens
-                                    (largest scores + most recent) stay, unchanged, in token order; pivot_rule,
-                                    weight_rule, sim_threshold and sigma are ignored, out_len = n_recent + n_heavy,
-                                    which must fit the capacity; set_id is -1 for dropped tokens and
-                                    set_start[s] = pivot[s] = the s-th kept token */
 };
 
 #define KVM_MAX_SEQ 65536
