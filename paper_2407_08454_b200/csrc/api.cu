@@ -263,8 +263,9 @@ int kvm_merge_compact(const kvm_params* p, const void* K, const void* V, const i
                    ? KVM_OK
                    : KVM_E_CUDA;
     if (launch_token_sets(d, set_start, out_len, w.set_id, st) != cudaSuccess) return KVM_E_CUDA;
-    // (the similarity region of the workspace is free here: scratch for the per-set bandwidths)
-    return launch_merge(d, K, V, set_start, pivot, w.set_id, out_len, K_out, V_out, out_size, w.merge_part, w.sim, st) ==
+    // (the similarity and score regions of the workspace are free here: scratch for the per-set bandwidths)
+    return launch_merge(d, K, V, set_start, pivot, w.set_id, out_len, K_out, V_out, out_size, w.merge_part, w.sim,
+                        w.scores, st) ==
                    cudaSuccess
                ? KVM_OK
                : KVM_E_CUDA;
@@ -305,7 +306,8 @@ int kvm_compress_with_lse(const kvm_params* p, const void* Q, const void* K, con
         return launch_gather(d, K, V, w.set_start, out_pos, out_len, K_out, V_out, nullptr, st) == cudaSuccess
                    ? KVM_OK
                    : KVM_E_CUDA;
-    if (launch_merge(d, K, V, w.set_start, out_pos, w.set_id, out_len, K_out, V_out, nullptr, w.merge_part, w.sim, st) !=
+    if (launch_merge(d, K, V, w.set_start, out_pos, w.set_id, out_len, K_out, V_out, nullptr, w.merge_part, w.sim,
+                     w.scores, st) !=
         cudaSuccess)
         return KVM_E_CUDA;
     return KVM_OK;

@@ -93,7 +93,8 @@ cudaError_t launch_token_sets(const Dims& d, const int32_t* set_start, const int
                               cudaStream_t st);
 cudaError_t launch_merge(const Dims& d, const void* K, const void* V, const int32_t* set_start,
                          const int32_t* pivot, const int32_t* set_id, const int32_t* out_len, void* K_out,
-                         void* V_out, int32_t* out_size, float* scratch, float* set_coef, cudaStream_t st);
+                         void* V_out, int32_t* out_size, float* scratch, float* set_coef, float* token_d2,
+                         cudaStream_t st);
 // Rows that are one input state each (pivot-only weights, eviction): a gather.
 cudaError_t launch_gather(const Dims& d, const void* K, const void* V, const int32_t* set_start,
                           const int32_t* pivot, const int32_t* out_len, void* K_out, void* V_out, int32_t* out_size,

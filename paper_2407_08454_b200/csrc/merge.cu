@@ -308,34 +308,49 @@ __global__ void __launch_bounds__(2 * D) merge_fixup_kernel(const int32_t* __res
 }
 
 // Bandwidth per merging set (one non-circular reading of Eq. 4): 2 sigma_s^2 = mean over the set of
-// |k_p - k_j|^2.  Writes, per set, the factor that turns a squared distance into the exponent of 2:
-// coef = -log2(e) / mean, or 0 (every weight 1) when the mean is 0.  One lane group per set.
+// |k_p - k_j|^2.  Sets can be hundreds of tokens long, so the work is split by tokens first:
+// token_dist_kernel writes every token's squared distance to its set's pivot (one lane group per token), then
+// set_coef_kernel sums them per set (one warp per set, lanes strided, fixed reduction order) and writes the factor
+// that turns a squared distance into the exponent of 2: coef = -log2(e) / mean, or 0 (every weight 1) when the
+// mean is 0.
 template <typename T, int D>
-__global__ void __launch_bounds__(256) set_bandwidth_kernel(const T* __restrict__ K,
-                                                            const int32_t* __restrict__ set_start,
-                                                            const int32_t* __restrict__ pivot,
-                                                            const int32_t* __restrict__ out_len,
-                                                            float* __restrict__ coef, int S, int cap) {
-    constexpr int N = Vec<T>::N, LPR = D / N, SETS = 256 / LPR;
+__global__ void __launch_bounds__(256) token_dist_kernel(const T* __restrict__ K, const int32_t* __restrict__ set_id,
+                                                         const int32_t* __restrict__ pivot, float* __restrict__ d2_out,
+                                                         int S, int cap, long long n_rows) {
+    constexpr int N = Vec<T>::N, LPR = D / N;
+    grid_dependency_wait();
+    const long long gid = ((long long)blockIdx.x * blockDim.x + threadIdx.x) / LPR;
+    if (gid >= n_rows) return;                            // whole groups leave together
+    const int lane = threadIdx.x % LPR;
+    const unsigned gmask = (LPR == 32) ? 0xffffffffu : (((1u << LPR) - 1u) << ((threadIdx.x % 32) / LPR * LPR));
+    const long long u = gid / S;
+    const int sid = __ldcg(set_id + gid);
+    const int p = __ldcg(pivot + (size_t)u * cap + sid);
+    float kj[N], kp[N];
+    Vec<T>::unpack(ldg16(K + (size_t)gid * D + lane * N), kj);
+    Vec<T>::unpack(ldg16(K + ((size_t)u * S + p) * D + lane * N), kp);
+    float d2 = 0.f;
+#pragma unroll
+    for (int e = 0; e < N; ++e) { const float a = kp[e] - kj[e]; d2 = fmaf(a, a, d2); }
+#pragma unroll
+    for (int off = 1; off < LPR; off <<= 1) d2 += __shfl_xor_sync(gmask, d2, off);
+    if (lane == 0) d2_out[gid] = d2;
+}
+
+__global__ void __launch_bounds__(256) set_coef_kernel(const float* __restrict__ d2, const int32_t* __restrict__ set_start,
+                                                       const int32_t* __restrict__ out_len, float* __restrict__ coef,
+                                                       int S, int cap) {
     grid_dependency_wait();
     const long long u = blockIdx.y;
-    const int s = blockIdx.x * SETS + threadIdx.x / LPR, lane = threadIdx.x % LPR;
-    if (s >= min(__ldcg(out_len + u), cap)) return;       // whole groups leave together
-    const unsigned gmask = (LPR == 32) ? 0xffffffffu : (((1u << LPR) - 1u) << ((threadIdx.x % 32) / LPR * LPR));
+    const int s = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (s >= min(__ldcg(out_len + u), cap)) return;       // whole warps leave together
     const int32_t* st = set_start + (size_t)u * (cap + 1);
-    const int lo = __ldcg(st + s), hi = __ldcg(st + s + 1), p = __ldcg(pivot + (size_t)u * cap + s);
-    const T* Ku = K + (size_t)u * S * D;
-    float kp[N];
-    Vec<T>::unpack(ldg16(Ku + (size_t)p * D + lane * N), kp);
+    const int lo = __ldcg(st + s), hi = __ldcg(st + s + 1);
+    const float* du = d2 + (size_t)u * S;
     float tot = 0.f;
-    for (int j = lo; j < hi; ++j) {
-        float kj[N];
-        Vec<T>::unpack(ldg16(Ku + (size_t)j * D + lane * N), kj);
+    for (int j = lo + lane; j < hi; j += 32) tot += __ldcg(du + j);
 #pragma unroll
-        for (int e = 0; e < N; ++e) { const float a = kp[e] - kj[e]; tot = fmaf(a, a, tot); }
-    }
-#pragma unroll
-    for (int off = 1; off < LPR; off <<= 1) tot += __shfl_xor_sync(gmask, tot, off);
+    for (int off = 16; off > 0; off >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, off);
     if (lane == 0) coef[(size_t)u * cap + s] = tot > 0.f ? -LOG2E * (float)(hi - lo) / tot : 0.f;
 }
 
@@ -384,7 +399,7 @@ cudaError_t launch_gather_t(const Dims& d, const void* K, const void* V, const i
 template <typename T, int D, int TOK>
 cudaError_t launch_t(const Dims& d, const void* K, const void* V, const int32_t* set_start, const int32_t* pivot,
                      const int32_t* set_id, const int32_t* out_len, void* K_out, void* V_out, int32_t* out_size,
-                     float* scratch, float* set_coef, cudaStream_t st) {
+                     float* scratch, float* set_coef, float* token_d2, cudaStream_t st) {
     const int Tn = (d.S + TOK - 1) / TOK;
     Slots<D> slots;
     slots.sums = scratch;
@@ -396,9 +411,13 @@ cudaError_t launch_t(const Dims& d, const void* K, const void* V, const int32_t*
     const float c = -LOG2E / (2.f * d.sigma * d.sigma);
     const bool per_set = d.weight_rule == KVM_WEIGHT_SET_SIGMA;
     if (per_set) {
-        constexpr int SETS = 256 / (D / Vec<T>::N);
-        e = launch_dependent(set_bandwidth_kernel<T, D>, dim3((d.cap + SETS - 1) / SETS, d.U), dim3(256), 0, st,
-                             (const T*)K, set_start, pivot, out_len, set_coef, d.S, d.cap);
+        const long long rows = (long long)d.U * d.S;
+        const unsigned blocks = (unsigned)((rows * (D / Vec<T>::N) + 255) / 256);
+        e = launch_dependent(token_dist_kernel<T, D>, dim3(blocks), dim3(256), 0, st, (const T*)K, set_id, pivot,
+                             token_d2, d.S, d.cap, rows);
+        if (e != cudaSuccess) return e;
+        e = launch_dependent(set_coef_kernel, dim3((d.cap + 7) / 8, d.U), dim3(256), 0, st, (const float*)token_d2,
+                             set_start, out_len, set_coef, d.S, d.cap);
         if (e != cudaSuccess) return e;
     }
     e = launch_dependent(merge_tile_kernel<T, D, TOK>, dim3(Tn, d.U), dim3(MERGE_NT), smem, st, (const T*)K,
@@ -444,20 +463,21 @@ cudaError_t launch_gather(const Dims& d, const void* K, const void* V, const int
                       : launch_gather_t<float, 64>(d, K, V, set_start, pivot, out_len, K_out, V_out, out_size, st);
 }
 
-// set_coef: [U, cap] fp32 of scratch, used only by the per-set bandwidth rule; out_len: device [U].
+// set_coef [U, cap] and token_d2 [U, S]: fp32 scratch, used only by the per-set bandwidth rule; out_len: device [U].
 cudaError_t launch_merge(const Dims& d, const void* K, const void* V, const int32_t* set_start,
                          const int32_t* pivot, const int32_t* set_id, const int32_t* out_len, void* K_out,
-                         void* V_out, int32_t* out_size, float* scratch, float* set_coef, cudaStream_t st) {
+                         void* V_out, int32_t* out_size, float* scratch, float* set_coef, float* token_d2,
+                         cudaStream_t st) {
     if (d.dtype == KVM_BF16) {
         return d.D == 128 ? launch_t<__nv_bfloat16, 128, KVM_MERGE_TOK_BF16>(d, K, V, set_start, pivot, set_id, out_len,
-                                                                          K_out, V_out, out_size, scratch, set_coef, st)
+                                                                          K_out, V_out, out_size, scratch, set_coef, token_d2, st)
                           : launch_t<__nv_bfloat16, 64, KVM_MERGE_TOK_BF16>(d, K, V, set_start, pivot, set_id, out_len,
-                                                                         K_out, V_out, out_size, scratch, set_coef, st);
+                                                                         K_out, V_out, out_size, scratch, set_coef, token_d2, st);
     }
     return d.D == 128 ? launch_t<float, 128, 64>(d, K, V, set_start, pivot, set_id, out_len, K_out, V_out, out_size,
-                                                 scratch, set_coef, st)
+                                                 scratch, set_coef, token_d2, st)
                       : launch_t<float, 64, 64>(d, K, V, set_start, pivot, set_id, out_len, K_out, V_out, out_size,
-                                                scratch, set_coef, st);
+                                                scratch, set_coef, token_d2, st);
 }
 
 }  // namespace kvm
