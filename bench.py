@@ -359,7 +359,7 @@ def main():
     e1.record(stream)
     barrier()
     ms_e2e = replicas.slowest_rank_ms(e0.elapsed_time(e1), dist, dev)
-    assert int(hlen.sum()) == out_rows or True
+    assert int(hlen.sum()) > 0, "the host path returned no rows"
     esz = 2 if cfg.dtype == "bf16" else 4
     h2d = (cfg.batch * cfg.n_q_heads + 2 * U) * cfg.seq * cfg.head_dim * esz
     d2h = 2 * U * comp.cap * cfg.head_dim * esz + U * 4 + U * comp.cap * 4
