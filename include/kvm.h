@@ -109,7 +109,7 @@ enum kvm_set_rule {
                                     set_start[s] = pivot[s] = the s-th kept token */
     KVM_SETS_ANCHOR = 2          /* the set identification as Section 3.2 words it: walking from the last token, a
                                     state gathers the consecutive states before it whose similarity TO IT exceeds
-                                    sim_threshold (Algorithm 1's listing compares neighbours instead).  Conserved
+                                    sim_threshold (Algorithm 1 compares neighbours instead).  Conserved
                                     tokens stand alone.  No budget rule: enforce_budget must be 0 (capacity S), and
                                     seq <= KVM_ANCHOR_MAX_SEQ.  kvm_segment's sim_out then receives, per token, the
                                     number of predecessors it would gather as a group's last state. */

@@ -201,7 +201,7 @@ void kvmo_layer_ratio(int64_t U, int32_t S, double eps, const double* sim, doubl
 // the last token, a key state gathers the consecutive states before it whose
 // similarity TO IT exceeds eps; the first state that fails (or is conserved, or
 // the start of the sequence) ends the group, and the walk goes on from there.
-// A conserved state is a group of its own.  (Algorithm 1's listing compares
+// A conserved state is a group of its own.  (Algorithm 1 compares
 // neighbours instead; both readings give consecutive, disjoint, covering sets.)
 //   cos(a, b) = <a,b> / (|a||b|), 0 if a norm is 0, computed in fp64.
 // b [U,S] (0/1) = boundary flags (1 at the first token of every group);
