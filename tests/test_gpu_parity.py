@@ -229,3 +229,36 @@ def test_host_entry_point_equals_the_device_path(B, Hq, Hkv, S, D, dtype):
                 assert torch.equal(hpos[u, :n], r.out_pos.cpu().view(B * Hkv, cap)[u, :n])
                 assert torch.equal(hK.view(B * Hkv, cap, D)[u, :n], r.K_out.cpu().view(B * Hkv, cap, D)[u, :n])
                 assert torch.equal(hV.view(B * Hkv, cap, D)[u, :n], r.V_out.cpu().view(B * Hkv, cap, D)[u, :n])
+
+
+def test_seeded_sweep_of_shapes_and_parameters():
+    """Thirty seeded draws of shape, dtype, budget, threshold, bandwidth and rules, each through the full parity
+    check: ragged lengths, single tiles, groups of 1 to 4 query heads, thresholds from permissive to strict."""
+    rng = np.random.default_rng(2024)
+    done = 0
+    while done < 30:
+        S = int(rng.integers(1, 900))
+        D = int(rng.choice([64, 128]))
+        Hkv = int(rng.integers(1, 4))
+        G = int(rng.choice([1, 2, 4]))
+        B = int(rng.integers(1, 3))
+        dtype = str(rng.choice(["bf16", "f32"]))
+        budget = float(rng.choice([0.35, 0.5, 0.75, 1.0]))
+        recent = float(rng.uniform(0.0, 0.2))
+        heavy = float(rng.uniform(0.0, 0.12))
+        eps = float(rng.uniform(0.3, 0.95))
+        sigma = float(rng.uniform(0.5, 8.0))
+        rho = float(rng.uniform(0.5, 0.98))
+        cap = int(np.floor(np.float32(budget) * S))
+        n_r, n_h = int(np.floor(np.float32(recent) * S)), int(np.floor(np.float32(heavy) * S))
+        if cap < 1 + n_r + 2 * n_h:
+            continue                                          # the host would refuse it (covered elsewhere)
+        cfg = si.CONFIGS["C1"].scaled(seq=S, head_dim=D, n_q_heads=Hkv * G, n_kv_heads=Hkv, batch=B, dtype=dtype,
+                                      budget=budget, rho=rho, seed=1000 + done)
+        d = si.make_layer(cfg)
+        rules = dict(pivot_rule=int(rng.integers(0, 2)), weight_rule=int(rng.choice([0, 1, 2, 3])))
+        case = Case(d["Q"], d["K"], d["V"], budget=budget, recent=recent, heavy=heavy, eps=eps, sigma=sigma,
+                    scale_v=bool(rng.integers(0, 2)), **rules)
+        rep = check_case(case)
+        print(done, (B, Hkv * G, Hkv, S, D, dtype), f"budget {budget} eps {eps:.2f} rules {rules}", rep.units_near_tie)
+        done += 1
