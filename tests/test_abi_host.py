@@ -103,3 +103,43 @@ def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "libkvm.so"))
     with pytest.raises(FileNotFoundError):
         binding.lib()
+
+
+def test_header_is_plain_c_and_links_from_c(lib, tmp_path):
+    """include/kvm.h must be usable from C: compile a small C99 program against it, link it with the
+    library, and run the host-only entry points (no device is touched)."""
+    import shutil
+    import subprocess
+    if shutil.which("gcc") is None:
+        pytest.skip("no C compiler")
+    src = tmp_path / "abi.c"
+    src.write_text(r'''
+#include <stdio.h>
+#include <string.h>
+#include "kvm.h"
+int main(void) {
+    kvm_params p;
+    memset(&p, 0, sizeof p);
+    p.batch = 1; p.n_q_heads = 32; p.n_kv_heads = 8; p.seq = 32768; p.head_dim = 128; p.dtype = KVM_BF16;
+    p.budget = 0.5f; p.recent_ratio = -1.f; p.heavy_ratio = -1.f; p.sim_threshold = 0.75f; p.sigma = 5.f;
+    p.causal = 1; p.scale_v_by_set_size = 1; p.enforce_budget = 1;
+    int32_t cap, nr, nh; size_t ws, host;
+    if (kvm_sizes(&p, &cap, &nr, &nh) != KVM_OK) return 1;
+    if (kvm_workspace_bytes(&p, &ws) != KVM_OK || kvm_host_staging_bytes(&p, &host) != KVM_OK) return 2;
+    p.head_dim = 96;
+    if (kvm_sizes(&p, &cap, &nr, &nh) != KVM_E_SHAPE) return 3;
+    printf("%d %d %d %zu %zu %d %s\n", (int)cap, (int)nr, (int)nh, ws, host, kvm_version(), kvm_status_string(KVM_E_SHAPE));
+    return 0;
+}
+''')
+    exe = tmp_path / "abi"
+    libdir = os.path.dirname(binding.LIB_PATH)
+    subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Werror", "-pedantic", "-I", os.path.join(ROOT, "include"),
+                           str(src), "-o", str(exe), "-L", libdir, "-l:libkvm.so", "-Wl,-rpath," + libdir])
+    out = subprocess.run([str(exe)], capture_output=True, text=True, timeout=120)
+    assert out.returncode == 0, out.stderr
+    cap, nr, nh, ws, host, ver = out.stdout.split()[:6]
+    assert (int(cap), int(nr), int(nh)) == (16384, 5570, 3932)
+    assert int(ws) == kvm.kvm_workspace_bytes(kvm.make_params(1, 32, 8, 32768, 128, kvm.KVM_BF16))
+    assert int(host) > int(ws) and int(ver) == kvm.kvm_version()
+    assert "shape" in out.stdout
