@@ -277,6 +277,13 @@ def main():
         "segment_gbs": (work["k_bytes"] + 3 * 4 * U * cfg.seq) / (t_segment * 1e-3) / 1e9,
         "score_both_passes_tflops": 2 * work["flops_per_score_pass"] / (t_score * 1e-3) / 1e12,
     }
+    # fraction of each step's own roofline (measured peaks): tensor for the score passes, HBM for the rest
+    kernels["roofline_frac"] = {
+        "score_both_passes": kernels["score_both_passes_tflops"] / peaks["bf16_tflops"],
+        "score_column_pass": achieved / peaks["bf16_tflops"],
+        "similarity_segment": kernels["segment_gbs"] / peaks["hbm_gbs"],
+        "merge_compact": kernels["merge_compact_gbs"] / peaks["hbm_gbs"],
+    }
     # the target's denominator: slower of score flops at tensor peak and total bytes at HBM bandwidth
     total_bytes = work["q_bytes"] + 2 * work["k_bytes"] + 2 * out_rows * cfg.head_dim * 2
     t_roof_ms = max(2 * work["flops_per_score_pass"] / (peaks["bf16_tflops"] * 1e12),
