@@ -6,7 +6,7 @@
 // Bandwidth-bound: every K and V row of the cache is read once per query head
 // (the G query heads of a KV head read the same rows within a short time, so
 // the repeats are L2 hits).  The rows of one (batch, query head) are split into
-// chunks of ATT_CHUNK rows, one block per chunk; inside a block a group of LPR
+// chunks sized so that the blocks fill the GPU in one wave, one block per chunk; inside a block a group of LPR
 // lanes owns a row at a time and keeps an online-softmax state (max, sum,
 // weighted V sum) in registers; groups, then chunks, are combined in a fixed
 // order, so results are reproducible.
@@ -16,10 +16,8 @@ namespace kvm {
 namespace {
 
 constexpr int ATT_NT = 256;
-#ifndef KVM_ATT_CHUNK
-#define KVM_ATT_CHUNK 256
-#endif
-constexpr int ATT_CHUNK = KVM_ATT_CHUNK;    // cache rows per block
+constexpr int ATT_MIN_CHUNK = 64;           // fewest cache rows a block is given (bounds the number of chunks)
+constexpr int ATT_BLOCKS_PER_SM = 4;        // resident blocks per SM (register-limited): the chunk count aims at one wave
 constexpr float LOG2E = 1.4426950408889634f;
 
 // Weight of a partial state with maximum m when the overall maximum is M (an empty state has m = -inf).
@@ -30,8 +28,8 @@ template <typename T, int D>
 __global__ void __launch_bounds__(ATT_NT) attend_partial_kernel(const T* __restrict__ q, const T* __restrict__ K,
                                                                 const T* __restrict__ V,
                                                                 const int32_t* __restrict__ len,
-                                                                float* __restrict__ part, int rows, int G, int Hq,
-                                                                int Hkv, float scale_log2e) {
+                                                                float* __restrict__ part, int rows, int chunk, int G,
+                                                                int Hq, int Hkv, float scale_log2e) {
     constexpr int N = Vec<T>::N, LPR = D / N, NGRP = ATT_NT / LPR;
     __shared__ float sm_m[NGRP], sm_l[NGRP];
     __shared__ __align__(16) float sm_acc[NGRP][D];
@@ -40,7 +38,7 @@ __global__ void __launch_bounds__(ATT_NT) attend_partial_kernel(const T* __restr
     const int b = bh / Hq, h = bh % Hq;
     const long long u = (long long)b * Hkv + h / G;
     const int n = len ? max(0, min(len[u], rows)) : rows;
-    const int r0 = split * ATT_CHUNK, r1 = min(r0 + ATT_CHUNK, n);
+    const int r0 = split * chunk, r1 = min(r0 + chunk, n);
     const int grp = threadIdx.x / LPR, lane = threadIdx.x % LPR;
     const unsigned gmask = (LPR == 32) ? 0xffffffffu : (((1u << LPR) - 1u) << ((threadIdx.x % 32) / LPR * LPR));
     const T* Ku = K + (size_t)u * rows * D;
@@ -167,9 +165,17 @@ __global__ void __launch_bounds__(D) perturbation_kernel(const float* __restrict
 template <typename T, int D>
 cudaError_t launch_t(const Dims& d, const void* q, const void* K, const void* V, int rows, const int32_t* len,
                      float* out, float* part, cudaStream_t st) {
-    const int nsplit = attend_splits(rows);
+    // as many chunks per head as keep every SM's resident blocks busy in a single wave, within the scratch bound
+    int dev = 0, sms = 0;
+    cudaError_t e0 = cudaGetDevice(&dev);
+    if (e0 == cudaSuccess) e0 = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e0 != cudaSuccess) return e0;
+    int want = (ATT_BLOCKS_PER_SM * sms) / (d.B * d.Hq);
+    want = want < 1 ? 1 : (want > attend_splits(rows) ? attend_splits(rows) : want);
+    const int chunk = (rows + want - 1) / want;
+    const int nsplit = (rows + chunk - 1) / chunk;
     attend_partial_kernel<T, D><<<dim3(nsplit, d.B * d.Hq), ATT_NT, 0, st>>>(
-        (const T*)q, (const T*)K, (const T*)V, len, part, rows, d.G, d.Hq, d.Hkv, d.scale * LOG2E);
+        (const T*)q, (const T*)K, (const T*)V, len, part, rows, chunk, d.G, d.Hq, d.Hkv, d.scale * LOG2E);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     return launch_dependent(attend_combine_kernel<D>, dim3(d.B * d.Hq), dim3(D), 0, st, (const float*)part, out, nsplit);
@@ -177,7 +183,8 @@ cudaError_t launch_t(const Dims& d, const void* q, const void* K, const void* V,
 
 }  // namespace
 
-int attend_splits(int rows) { return (rows + ATT_CHUNK - 1) / ATT_CHUNK; }
+// Upper bound on the chunks per head (what the scratch is sized for).
+int attend_splits(int rows) { return (rows + ATT_MIN_CHUNK - 1) / ATT_MIN_CHUNK; }
 
 size_t attend_scratch_floats(const Dims& d) { return (size_t)d.B * d.Hq * attend_splits(d.S) * (d.D + 2); }
 
