@@ -147,6 +147,15 @@ int kvm_score(const kvm_params* p, const void* Q, const void* K, const float* ls
               float* scores, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * The row pass of kvm_score alone: the natural-log row log-sum-exp of the scaled causal logits (Eq. 1's softmax
+ * normaliser), lse_out [batch, n_q_heads, S] fp32, written.  It is what kvm_score and kvm_compress_with_lse accept
+ * as lse_in, so a caller that compresses the same layer several times (other budgets, thresholds or rules) pays
+ * for the row pass once.
+ */
+int kvm_row_lse(const kvm_params* p, const void* Q, const void* K, float* lse_out, void* ws, size_t ws_bytes,
+                void* cuda_stream);
+
+/*
  * Merging-set identification and pivots (Eq. 2, Algorithm 1, Definition 4.1, Eq. 6).
  *   K [batch, n_kv_heads, S, D]; scores [batch, n_kv_heads, S] fp32.
  *   Conserved tokens: the last n_recent positions and, among the others, the

@@ -23,7 +23,7 @@ KVM_PIVOT_MAX_SCORE, KVM_PIVOT_LAST, KVM_PIVOT_KEY = 0, 1, 2
 KVM_WEIGHT_GAUSSIAN, KVM_WEIGHT_AVERAGE, KVM_WEIGHT_PIVOT_ONLY, KVM_WEIGHT_SET_SIGMA = 0, 1, 2, 3
 KVM_SETS_ADJACENT, KVM_SETS_CONSERVED_ONLY, KVM_SETS_ANCHOR = 0, 1, 2
 EXPORTS = (
-    "kvm_sizes", "kvm_workspace_bytes", "kvm_score", "kvm_segment", "kvm_merge_compact", "kvm_compress",
+    "kvm_sizes", "kvm_workspace_bytes", "kvm_score", "kvm_row_lse", "kvm_segment", "kvm_merge_compact", "kvm_compress",
     "kvm_compress_with_lse",
     "kvm_host_staging_bytes", "kvm_compress_host", "kvm_score_static", "kvm_layer_ratio", "kvm_attend",
     "kvm_output_perturbation", "kvm_status_string",
@@ -145,6 +145,11 @@ def kvm_host_staging_bytes(p: KvmParams) -> int:
 def kvm_score(p: KvmParams, Q, K, lse_in, scores, ws, stream=None) -> None:
     _check(lib().kvm_score(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(lse_in), _ptr(scores), _ptr(ws),
                            ctypes.c_size_t(ws.numel() * ws.element_size()), _stream(stream)), "kvm_score")
+
+
+def kvm_row_lse(p: KvmParams, Q, K, lse_out, ws, stream=None) -> None:
+    _check(lib().kvm_row_lse(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(lse_out), _ptr(ws),
+                             ctypes.c_size_t(ws.numel() * ws.element_size()), _stream(stream)), "kvm_row_lse")
 
 
 def kvm_score_static(p: KvmParams, Q, K, scores, stream=None) -> None:

@@ -176,6 +176,28 @@ int kvm_score(const kvm_params* p, const void* Q, const void* K, const float* ls
                                                                                                     : KVM_E_CUDA;
 }
 
+int kvm_row_lse(const kvm_params* p, const void* Q, const void* K, float* lse_out, void* ws, size_t ws_bytes,
+                void* cuda_stream) {
+    Dims d;
+    int rc = derive(p, d);
+    if (rc != KVM_OK) return rc;
+    if (!Q || !K || !lse_out) return KVM_E_NULL;
+    if (misaligned(Q) || misaligned(K) || misaligned(lse_out)) return KVM_E_ALIGN;
+    Workspace w;
+    if ((rc = check_ws(d, ws, ws_bytes, w)) != KVM_OK) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (d.dtype == KVM_BF16)
+        return launch_score_tc(d, Q, K, nullptr, w.lse, nullptr, nullptr, st, nullptr, lse_out) == cudaSuccess
+                   ? KVM_OK
+                   : KVM_E_CUDA;
+    // fp32 path: its row pass leaves the natural-log lse in the workspace as it is
+    if (launch_score_simt(d, Q, K, nullptr, w.lse, nullptr, st) != cudaSuccess) return KVM_E_CUDA;
+    return cudaMemcpyAsync(lse_out, w.lse, (size_t)d.B * d.Hq * d.S * sizeof(float), cudaMemcpyDeviceToDevice, st) ==
+                   cudaSuccess
+               ? KVM_OK
+               : KVM_E_CUDA;
+}
+
 int kvm_segment(const kvm_params* p, const void* K, const float* scores, int32_t* set_id, int32_t* set_start,
                 int32_t* pivot, int32_t* out_len, float* sim_out, kvm_stats* stats, void* ws, size_t ws_bytes,
                 void* cuda_stream) {

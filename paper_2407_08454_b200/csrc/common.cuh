@@ -80,7 +80,8 @@ cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, si
 cudaError_t launch_score_simt(const Dims& d, const void* Q, const void* K, const float* lse_in, float* lse_ws,
                               float* scores, cudaStream_t st);
 cudaError_t launch_score_tc(const Dims& d, const void* Q, const void* K, const float* lse_in, float* lse_ws,
-                            float* scores, kvm_stats* stats, cudaStream_t st, float* sim_out = nullptr);
+                            float* scores, kvm_stats* stats, cudaStream_t st, float* sim_out = nullptr,
+                            float* lse_out = nullptr);
 size_t score_tc_scratch_bytes_per_row();
 cudaError_t launch_similarity(const Dims& d, const void* K, float* sim, cudaStream_t st);
 cudaError_t launch_segment(const Dims& d, const float* scores, const float* sim, int32_t* set_id,

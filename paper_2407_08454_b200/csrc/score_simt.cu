@@ -174,16 +174,18 @@ cudaError_t launch_score_simt(const Dims& d, const void* Q, const void* K, const
                                                                          d.Hq, d.G, d.S, d.D, scale2);
             lse = lse_ws;
         }
-        colsum_simt_kernel<float><<<dim3(nT, d.U), 256, 0, st>>>((const float*)Q, (const float*)K, lse, scores,
-                                                                 d.Hq, d.G, d.S, d.D, scale2);
+        if (scores)
+            colsum_simt_kernel<float><<<dim3(nT, d.U), 256, 0, st>>>((const float*)Q, (const float*)K, lse, scores,
+                                                                     d.Hq, d.G, d.S, d.D, scale2);
     } else {
         if (!lse_in) {
             lse_simt_kernel<__nv_bfloat16><<<dim3(nT, d.B * d.Hq), 256, 0, st>>>(
                 (const __nv_bfloat16*)Q, (const __nv_bfloat16*)K, lse_ws, d.Hq, d.G, d.S, d.D, scale2);
             lse = lse_ws;
         }
-        colsum_simt_kernel<__nv_bfloat16><<<dim3(nT, d.U), 256, 0, st>>>(
-            (const __nv_bfloat16*)Q, (const __nv_bfloat16*)K, lse, scores, d.Hq, d.G, d.S, d.D, scale2);
+        if (scores)
+            colsum_simt_kernel<__nv_bfloat16><<<dim3(nT, d.U), 256, 0, st>>>(
+                (const __nv_bfloat16*)Q, (const __nv_bfloat16*)K, lse, scores, d.Hq, d.G, d.S, d.D, scale2);
     }
     return cudaGetLastError();
 }

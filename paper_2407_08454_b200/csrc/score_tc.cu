@@ -660,10 +660,22 @@ __global__ void __launch_bounds__(256) lse_split_kernel(const float* __restrict_
     dst[1] = make_uint4(0u, 0u, 0u, 0u);
 }
 
+// The row pass's side tensor back to a natural-log lse per query row: lse = -(hi + mid + lo) * scale2 * ln 2.
+__global__ void __launch_bounds__(256) side_to_lse_kernel(const __nv_bfloat16* __restrict__ side, float* __restrict__ lse,
+                                                          long long rows, float neg_scale2_ln2) {
+    grid_dependency_wait();
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= rows) return;
+    const uint2 raw = __ldcg(reinterpret_cast<const uint2*>(side + (size_t)i * PCH));
+    const float hi = __uint_as_float(raw.x << 16), mid = __uint_as_float(raw.x & 0xffff0000u);
+    const float lo = __uint_as_float(raw.y << 16);
+    lse[i] = ((hi + mid) + lo) * neg_scale2_ln2;
+}
+
 template <int KCH>
 cudaError_t launch_t(const Dims& d, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mp,
                      const float* lse_in, __nv_bfloat16* side, float* scores, kvm_stats* stats, cudaStream_t st,
-                     const __nv_bfloat16* Ksim, float* sim_out) {
+                     const __nv_bfloat16* Ksim, float* sim_out, float* lse_out) {
     const size_t smem = 1024 + (size_t)(2 + 2 * NSTAGE) * KCH * TILE * 128 + (size_t)(2 * NSTAGE + 1) * PTILE_BYTES +
                         sizeof(Shared);
     cudaError_t e = cudaFuncSetAttribute(score_tc_kernel<KCH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -686,6 +698,13 @@ cudaError_t launch_t(const Dims& d, const CUtensorMap& mq, const CUtensorMap& mk
     }
     const bool sim_in_pass2 = lse_in != nullptr;      // no row pass: the column pass's spare warps do it
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    if (lse_out) {                                    // the caller wants the row pass's result in the clear
+        const long long rows = (long long)d.B * d.Hq * d.S;
+        e = launch_dependent(side_to_lse_kernel, dim3((unsigned)((rows + 255) / 256)), dim3(256), 0, st,
+                             (const __nv_bfloat16*)side, lse_out, rows, -scale2 * 0.6931471805599453f);
+        if (e != cudaSuccess) return e;
+    }
+    if (!scores) return cudaSuccess;                  // row pass only
     const long long items = (long long)d.U * T;
     const int grid = (int)(items < sms ? items : sms);
     return launch_dependent(score_tc_kernel<KCH>, dim3(grid), dim3(NTHREADS), smem, st, mq, mk, mp,
@@ -700,16 +719,17 @@ size_t score_tc_scratch_bytes_per_row() { return (size_t)PCH * 2; }
 
 // sim_out (nullable): when given, the spare warps of the row pass (of the column pass when lse_in replaces
 // the row pass) also write the neighbour-key similarities [U,S] there, so the caller needs no similarity kernel.
+// scores may be NULL (row pass only); lse_out (nullable) receives the natural-log row log-sum-exp [B,Hq,S].
 cudaError_t launch_score_tc(const Dims& d, const void* Q, const void* K, const float* lse_in, float* lse_ws,
-                            float* scores, kvm_stats* stats, cudaStream_t st, float* sim_out) {
+                            float* scores, kvm_stats* stats, cudaStream_t st, float* sim_out, float* lse_out) {
     CUtensorMap mq, mk, mp;
     __nv_bfloat16* side = reinterpret_cast<__nv_bfloat16*>(lse_ws);
     if (!make_map(&mq, Q, d.B * d.Hq, d.S, d.D) || !make_map(&mk, K, d.B * d.Hkv, d.S, d.D) ||
         !make_map_side(&mp, side, d.B * d.Hq, d.S))
         return cudaErrorNotSupported;
     const __nv_bfloat16* Ks = reinterpret_cast<const __nv_bfloat16*>(K);
-    return d.D == 128 ? launch_t<2>(d, mq, mk, mp, lse_in, side, scores, stats, st, Ks, sim_out)
-                      : launch_t<1>(d, mq, mk, mp, lse_in, side, scores, stats, st, Ks, sim_out);
+    return d.D == 128 ? launch_t<2>(d, mq, mk, mp, lse_in, side, scores, stats, st, Ks, sim_out, lse_out)
+                      : launch_t<1>(d, mq, mk, mp, lse_in, side, scores, stats, st, Ks, sim_out, lse_out);
 }
 
 }  // namespace kvm

@@ -94,6 +94,26 @@ def test_lse_in_skips_the_row_pass_and_matches():
     assert score_excess(out.cpu().numpy(), ref) <= 1.0
 
 
+@pytest.mark.parametrize("dtype,S,D", [("bf16", 900, 128), ("f32", 512, 64), ("bf16", 300, 64)])
+def test_row_lse_matches_the_checker_and_feeds_the_column_pass(dtype, S, D):
+    from oracle import kvmo
+    cfg = si.CONFIGS["C1"].scaled(seq=S, head_dim=D, n_q_heads=4, n_kv_heads=2, dtype=dtype, seed=12)
+    d = si.make_layer(cfg)
+    _, ref_lse = kvmo.scores(d["Q"], d["K"], want_lse=True)
+    p = Case(d["Q"], d["K"], d["V"]).params()
+    ws = torch.empty(kvm.kvm_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+    Q, K = d["Q"].cuda(), d["K"].cuda()
+    lse = torch.full((1, 4, S), float("nan"), device="cuda")
+    kvm.kvm_row_lse(p, Q, K, lse, ws)
+    # fp32 accumulation of the logits and an approximate exp2 / log2: a few 1e-5 on values of order 10
+    assert np.abs(lse.cpu().numpy() - ref_lse).max() <= 2e-4
+    a = torch.empty(1, 2, S, device="cuda")
+    b = torch.empty(1, 2, S, device="cuda")
+    kvm.kvm_score(p, Q, K, None, a, ws)
+    kvm.kvm_score(p, Q, K, lse, b, ws)
+    np.testing.assert_allclose(b.cpu().numpy(), a.cpu().numpy(), rtol=2e-5, atol=1e-7)   # same lse, re-split to bf16 terms
+
+
 @pytest.mark.parametrize("dtype,S,D", [("bf16", 900, 128), ("f32", 512, 64)])
 def test_compress_with_caller_lse_matches_the_checker(dtype, S, D):
     from oracle import kvmo
