@@ -195,6 +195,8 @@ int kvm_merge_compact(const kvm_params* p, const void* K, const void* V,
 /*
  * The whole path for one layer: kvm_score, kvm_segment, kvm_merge_compact chained
  * on the stream with intermediates in the workspace.
+ * (No allocation, no synchronisation, no host-side state: the call can be captured
+ * into a CUDA graph and replayed.)
  *   out_pos    [U, cap] i32   pivot token index of each output row (ascending)
  *   scores_out NULL or [U, S] fp32
  *   stats      NULL or device kvm_stats

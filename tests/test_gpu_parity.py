@@ -282,3 +282,29 @@ def test_seeded_sweep_of_shapes_and_parameters():
         rep = check_case(case)
         print(done, (B, Hkv * G, Hkv, S, D, dtype), f"budget {budget} eps {eps:.2f} rules {rules}", rep.units_near_tie)
         done += 1
+
+
+def test_compress_replays_from_a_cuda_graph():
+    # nothing in kvm_compress allocates or synchronises, so the call can be captured once and replayed
+    cfg = si.CONFIGS["C1"].scaled(seq=1024, n_q_heads=8, n_kv_heads=4, seed=77)
+    d = {k: v.cuda() for k, v in si.make_layer(cfg).items()}
+    p = kvm.make_params(1, 8, 4, 1024, 128, torch.bfloat16)
+    c = kvm.Compressor(p)
+    c(d["Q"], d["K"], d["V"])
+    torch.cuda.synchronize()
+    ref = [t.clone() for t in (c.K_out, c.V_out, c.out_len, c.out_pos)]
+    for t in (c.K_out, c.V_out, c.out_len, c.out_pos):
+        t.zero_()
+    g, s = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+    with torch.cuda.stream(s), torch.cuda.graph(g, stream=s):
+        kvm.kvm_compress(p, d["Q"], d["K"], d["V"], c.K_out, c.V_out, c.out_len, c.out_pos, None, None, c.ws)
+    torch.cuda.synchronize()
+    assert int(c.out_len.sum()) == 0                 # capture enqueues nothing
+    for _ in range(2):
+        g.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(c.out_len, ref[2])
+    for u in range(4):
+        n = int(ref[2][0, u])
+        assert torch.equal(c.K_out[0, u, :n], ref[0][0, u, :n]) and torch.equal(c.V_out[0, u, :n], ref[1][0, u, :n])
+        assert torch.equal(c.out_pos[0, u, :n], ref[3][0, u, :n])
