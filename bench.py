@@ -270,6 +270,16 @@ def main():
         "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"], "traffic": NCU_TRAFFIC_BYTES_COLUMN_PASS,
         "peak_source": peaks["source"] + " burst bf16",
     }
+    # the same kernel against the unit that actually limits it: one exponential per causal logit on the
+    # special-function units (16 results per clock per SM)
+    exps_per_pass = cfg.batch * cfg.n_q_heads * cfg.seq * (cfg.seq + 1) / 2.0
+    sfu_peak = 16.0 * torch.cuda.get_device_properties(dev).multi_processor_count * (clk.max_mhz or 1965) * 1e6
+    roofline_sfu = {
+        "kernel": roofline["kernel"], "bound": "alu", "unit": "Gexp/s",
+        "achieved": exps_per_pass / (t_colsum * 1e-3) / 1e9, "peak": sfu_peak / 1e9,
+        "frac": exps_per_pass / (t_colsum * 1e-3) / sfu_peak,
+        "peak_source": "16 ex2 per clock per SM x SM count x maximum SM clock",
+    }
     kernels = {
         "score_both_passes_ms": t_score, "score_column_pass_ms": t_colsum, "similarity_segment_ms": t_segment,
         "merge_compact_ms": t_merge,
@@ -399,7 +409,7 @@ def main():
                        "l2": f"inputs larger than L2: {N_BUFFERS} rotating layer input sets of 100.7 MB",
                        "parallelism": f"replicas x{world} (independent layers per GPU, no collective)"},
             "clocks": clk.summary(), "e2e": e2e, "gpu_launches": 5 * args.steps,
-            "roofline": roofline, "kernels": kernels, "extras": extras,
+            "roofline": roofline, "roofline_sfu": roofline_sfu, "kernels": kernels, "extras": extras,
             "path_roofline": {"roof_ms_per_step": t_roof_ms, "frac": e2e_frac,
                               "note": "slower of 2 score passes at bf16 peak and total bytes at HBM peak"},
             "cpu_baseline": cpu,
