@@ -54,7 +54,8 @@ def build(force: bool = False, verbose: bool = False, extra=()) -> str:
     if failed:
         raise RuntimeError("nvcc failed")
     tmp = LIB + f".tmp{os.getpid()}"
-    subprocess.check_call([nvcc, "-shared", "-o", tmp, *objs, "-lcudart_static", "-ldl", "-lrt", "-lpthread"])
+    subprocess.check_call([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", tmp, *objs,
+                           "-lcudart_static", "-ldl", "-lrt", "-lpthread"])
     os.replace(tmp, LIB)
     return LIB
 
