@@ -364,13 +364,14 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const T* __restrict__ 
                                                           T* __restrict__ V_out, int32_t* __restrict__ out_size,
                                                           int S, int cap, int scale_v, int singletons) {
     constexpr int N = Vec<T>::N, LPR = D / N, ROWS = 256 / LPR / 2;
+    grid_dependency_wait();     // sets and pivots come from the kernel before this one
     const long long u = blockIdx.y;
     const int g = threadIdx.x / LPR, lane = threadIdx.x % LPR;
     const int s = blockIdx.x * ROWS + (g >> 1), which = g & 1;
-    if (s >= min(out_len[u], cap)) return;
-    const int p = __ldg(pivot + (size_t)u * cap + s);
+    if (s >= min(__ldcg(out_len + u), cap)) return;
+    const int p = __ldcg(pivot + (size_t)u * cap + s);
     const int32_t* st = set_start + (size_t)u * (cap + 1);
-    const int n = singletons ? 1 : __ldg(st + s + 1) - __ldg(st + s);
+    const int n = singletons ? 1 : __ldcg(st + s + 1) - __ldcg(st + s);
     const T* src = (which ? V : K) + ((size_t)u * S + p) * D + lane * N;
     T* dst = (which ? V_out : K_out) + ((size_t)u * cap + s) * D + lane * N;
     uint4 r = ldg16(src);
@@ -390,10 +391,9 @@ cudaError_t launch_gather_t(const Dims& d, const void* K, const void* V, const i
                             const int32_t* pivot, const int32_t* out_len, void* K_out, void* V_out,
                             int32_t* out_size, cudaStream_t st) {
     constexpr int ROWS = 256 / (D / Vec<T>::N) / 2;
-    gather_rows_kernel<T, D><<<dim3((d.cap + ROWS - 1) / ROWS, d.U), 256, 0, st>>>(
-        (const T*)K, (const T*)V, set_start, pivot, out_len, (T*)K_out, (T*)V_out, out_size, d.S, d.cap, d.scale_v,
-        d.set_rule == KVM_SETS_CONSERVED_ONLY ? 1 : 0);
-    return cudaGetLastError();
+    return launch_dependent(gather_rows_kernel<T, D>, dim3((d.cap + ROWS - 1) / ROWS, d.U), dim3(256), 0, st,
+                            (const T*)K, (const T*)V, set_start, pivot, out_len, (T*)K_out, (T*)V_out, out_size, d.S,
+                            d.cap, d.scale_v, d.set_rule == KVM_SETS_CONSERVED_ONLY ? 1 : 0);
 }
 
 template <typename T, int D, int TOK>
