@@ -78,7 +78,7 @@ typedef struct kvm_params {
     int32_t pivot_rule;          /* kvm_pivot_rule */
     int32_t weight_rule;         /* kvm_weight_rule */
     int32_t set_rule;            /* kvm_set_rule */
-    const float* pivot_key;      /* device [U, S] fp32, finite; read only when pivot_rule == KVM_PIVOT_KEY, else NULL */
+    const float* pivot_key;      /* device [U, S] fp32, finite, 4-byte aligned; read only when pivot_rule == KVM_PIVOT_KEY, else NULL */
 } kvm_params;
 
 /* How the pivot of a merging set is chosen. */
@@ -279,9 +279,10 @@ int kvm_output_perturbation(const kvm_params* p, const void* q, const void* K, c
  * not acceptable -- and that has no spare buffer to lend as a workspace.
  *
  * Instead of a caller workspace, the row log-sum-exp scratch lives in a fixed
- * array built into the library image: KVM_STATIC_SCORE_ROWS floats (4 MiB) plus
- * 256 bytes of counters.  Every GPU that loads the library holds that array
- * until the process exits, whether or not this function is ever called.
+ * array built into the library image: KVM_STATIC_SCORE_ROWS floats (4 MiB).  Every
+ * GPU on which the CUDA runtime loads the library's device code holds that array
+ * from then (at the latest from this function's first call there) until the process
+ * exits, whether or not the function is called again.
  *
  *   - Same Q, K, scores and stream arguments as kvm_score; no lse_in, no ws.
  *   - batch * n_q_heads * seq must not exceed KVM_STATIC_SCORE_ROWS for fp32 tensors and
@@ -291,10 +292,11 @@ int kvm_output_perturbation(const kvm_params* p, const void* q, const void* K, c
  *     one-time host-side set-up, done with that device current).  Make that first
  *     call outside any stream capture.
  *   - All calls on one device share the one array and it keeps whatever the last
- *     call left there.  The function re-initialises the part that must start at
- *     zero on every call, but two calls whose kernels overlap on the GPU (different
- *     streams, no ordering between them) race on it and give wrong scores: order
- *     such calls on one stream or with events.
+ *     call left there.  Nothing in it has to start at zero (the row pass rewrites
+ *     every row before the column pass reads it), but two calls whose kernels
+ *     overlap on the GPU (different streams, no ordering between them) write and
+ *     read the same rows and give wrong scores: order such calls on one stream or
+ *     with events.
  *   - Calls no cudaMalloc/cudaFree and no allocating library routine.
  */
 #define KVM_STATIC_SCORE_ROWS (1 << 20)

@@ -21,20 +21,27 @@ def sources():
     return sorted(glob.glob(os.path.join(CSRC, "*.cu")))
 
 
-def _stale() -> bool:
-    if not os.path.exists(LIB):
+# A second library for the test of the give-up path of the bounded device waits: the same sources with a short
+# wait limit and a producer that leaves out one stage, so that a wait runs out, the kernel returns and reports
+# it.  It is never loaded by the package itself.
+WAITTEST_LIB = os.path.join(_PKG, "libkvm_waittest.so")
+WAITTEST_FLAGS = ("-DKVM_TEST_WAIT_LIMIT_CLOCKS=4000000ll", "-DKVM_TEST_DROP_B_STAGE=3")
+
+
+def _stale(lib: str = LIB) -> bool:
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     deps = sources() + glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(_ROOT, "include", "*.h"))
     return any(os.path.getmtime(f) > t for f in deps)
 
 
-def build(force: bool = False, verbose: bool = False, extra=()) -> str:
+def build(force: bool = False, verbose: bool = False, extra=(), lib: str = LIB) -> str:
     """Compile every .cu under csrc/ into one shared library.  Returns its path."""
-    if not force and not _stale():
-        return LIB
+    if not force and not _stale(lib):
+        return lib
     nvcc = os.environ.get("NVCC", "nvcc")
-    objdir = os.path.join(_PKG, "_build")
+    objdir = os.path.join(_PKG, "_build" + os.path.basename(lib)[len("libkvm"):-len(".so")])
     os.makedirs(objdir, exist_ok=True)
     procs = []
     objs = []
@@ -53,11 +60,16 @@ def build(force: bool = False, verbose: bool = False, extra=()) -> str:
         failed |= p.returncode != 0
     if failed:
         raise RuntimeError("nvcc failed")
-    tmp = LIB + f".tmp{os.getpid()}"
+    tmp = lib + f".tmp{os.getpid()}"
     subprocess.check_call([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", tmp, *objs,
                            "-lcudart_static", "-ldl", "-lrt", "-lpthread"])
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, lib)
+    return lib
+
+
+def build_waittest(force: bool = False) -> str:
+    """The test-only library with a short wait limit and a dropped producer stage (see WAITTEST_FLAGS)."""
+    return build(force=force, extra=WAITTEST_FLAGS, lib=WAITTEST_LIB)
 
 
 if __name__ == "__main__":

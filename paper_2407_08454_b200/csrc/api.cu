@@ -49,7 +49,8 @@ int derive(const kvm_params* p, Dims& d) {
         if ((long long)d.cap < (long long)d.n_r + d.n_h) return KVM_E_PARAM;   // the kept tokens must fit
     } else {
         if (d.pivot_rule == KVM_PIVOT_KEY && !d.pivot_key) return KVM_E_NULL;
-        if (d.pivot_rule == KVM_PIVOT_KEY && ((uintptr_t)d.pivot_key & 15u)) return KVM_E_ALIGN;
+        // (pivot_key is read with scalar loads: no alignment beyond a float's is asked of it)
+        if (d.pivot_rule == KVM_PIVOT_KEY && ((uintptr_t)d.pivot_key & 3u)) return KVM_E_ALIGN;
         // the forced cuts alone (first token, recent window, each heavy hitter and its right neighbour) must fit
         if (d.enforce && (long long)d.cap < 1LL + d.n_r + 2LL * d.n_h) return KVM_E_PARAM;
     }
@@ -66,7 +67,6 @@ inline size_t score_row_bytes(const Dims& d) {
 }
 
 struct Workspace {
-    int* counters;      // 64 ints
     float* lse;         // row-pass output: [B,Hq,S] fp32 (fp32 path) or [B,Hq,S,16] bf16 side tensor (bf16 path)
     float* scores;      // [U,S]
     float* sim;         // [U,S]
@@ -81,7 +81,6 @@ Workspace carve(const Dims& d, void* base) {
     Workspace w;
     size_t off = 0;
     auto take = [&](size_t n) { size_t o = off; off += align_up(n); return (char*)base + o; };
-    w.counters = (int*)take(64 * sizeof(int));
     w.lse = (float*)take((size_t)d.B * d.Hq * d.S * score_row_bytes(d));
     w.scores = (float*)take((size_t)d.U * d.S * sizeof(float));
     w.sim = (float*)take((size_t)d.U * d.S * sizeof(float));
@@ -287,7 +286,7 @@ int kvm_merge_compact(const kvm_params* p, const void* K, const void* V, const i
     if (launch_token_sets(d, set_start, out_len, w.set_id, st) != cudaSuccess) return KVM_E_CUDA;
     // (the similarity and score regions of the workspace are free here: scratch for the per-set bandwidths)
     return launch_merge(d, K, V, set_start, pivot, w.set_id, out_len, K_out, V_out, out_size, w.merge_part, w.sim,
-                        w.scores, st) ==
+                        w.scores, nullptr, st) ==
                    cudaSuccess
                ? KVM_OK
                : KVM_E_CUDA;
@@ -329,7 +328,7 @@ int kvm_compress_with_lse(const kvm_params* p, const void* Q, const void* K, con
                    ? KVM_OK
                    : KVM_E_CUDA;
     if (launch_merge(d, K, V, w.set_start, out_pos, w.set_id, out_len, K_out, V_out, nullptr, w.merge_part, w.sim,
-                     w.scores, st) !=
+                     w.scores, stats, st) !=
         cudaSuccess)
         return KVM_E_CUDA;
     return KVM_OK;
@@ -418,34 +417,60 @@ int kvm_compress_host(const kvm_params* p, const void* Q, const void* K, const v
     const int nch = d.U < kHostChunksMax ? d.U : kHostChunksMax;
     const int per = (d.U + nch - 1) / nch;
     auto ok = [](cudaError_t err) { return err == cudaSuccess; };
-    if (!ok(cudaEventRecord(hp->start, st)) || !ok(cudaStreamWaitEvent(hp->compute, hp->start, 0)) ||
-        !ok(cudaStreamWaitEvent(hp->d2h, hp->start, 0)))
-        return KVM_E_CUDA;
-    for (int c = 0, u0 = 0; u0 < d.U; ++c, u0 += per) {
-        const int nu = (d.U - u0 < per) ? d.U - u0 : per;
-        kvm_params pc = *p;                      // the group as a layer of its own: one batch entry, nu KV heads
+    // a group of units as a layer of its own: one batch entry, nu KV heads
+    auto group_params = [&](int u0, int nu) {
+        kvm_params pc = *p;
         pc.batch = 1;
         pc.n_kv_heads = nu;
         pc.n_q_heads = nu * d.G;
         if (pc.pivot_key) pc.pivot_key += (size_t)u0 * d.S;
+        return pc;
+    };
+    // every group is validated before anything is enqueued, so a refusal leaves no copy in flight
+    for (int u0 = 0; u0 < d.U; u0 += per) {
+        const kvm_params pc = group_params(u0, (d.U - u0 < per) ? d.U - u0 : per);
+        Dims dc;
+        size_t need_c = 0;
+        if ((rc = derive(&pc, dc)) != KVM_OK) return rc;
+        if ((rc = kvm_workspace_bytes(&pc, &need_c)) != KVM_OK) return rc;
+        if (need_c > ws_bytes) return KVM_E_WORKSPACE;
+    }
+    if (!ok(cudaEventRecord(hp->start, st)) || !ok(cudaStreamWaitEvent(hp->compute, hp->start, 0)) ||
+        !ok(cudaStreamWaitEvent(hp->d2h, hp->start, 0)))
+        return KVM_E_CUDA;
+    // From here on work is in flight on the library's streams: whatever happens, the caller's stream is made
+    // to wait for all of it before the call returns, so that an error return never leaves copies writing the
+    // caller's buffers behind its back.
+    int status = KVM_OK;
+    for (int c = 0, u0 = 0; u0 < d.U && status == KVM_OK; ++c, u0 += per) {
+        const int nu = (d.U - u0 < per) ? d.U - u0 : per;
+        const kvm_params pc = group_params(u0, nu);
         if (!ok(cudaMemcpyAsync(dQ + rowQ * u0, (const char*)Q + rowQ * u0, rowQ * nu, cudaMemcpyHostToDevice, st)) ||
             !ok(cudaMemcpyAsync(dK + rowK * u0, (const char*)K + rowK * u0, rowK * nu, cudaMemcpyHostToDevice, st)) ||
             !ok(cudaMemcpyAsync(dV + rowK * u0, (const char*)V + rowK * u0, rowK * nu, cudaMemcpyHostToDevice, st)) ||
-            !ok(cudaEventRecord(hp->h2d[c], st)) || !ok(cudaStreamWaitEvent(hp->compute, hp->h2d[c], 0)))
-            return KVM_E_CUDA;
+            !ok(cudaEventRecord(hp->h2d[c], st)) || !ok(cudaStreamWaitEvent(hp->compute, hp->h2d[c], 0))) {
+            status = KVM_E_CUDA;
+            break;
+        }
         rc = kvm_compress(&pc, dQ + rowQ * u0, dK + rowK * u0, dV + rowK * u0, dKo + rowO * u0, dVo + rowO * u0,
                           (int32_t*)dL + u0, (int32_t*)(dP + rowP * u0), nullptr, nullptr, ws, ws_bytes, hp->compute);
-        if (rc != KVM_OK) return rc;
+        if (rc != KVM_OK) {
+            status = rc;
+            break;
+        }
         if (!ok(cudaEventRecord(hp->done[c], hp->compute)) || !ok(cudaStreamWaitEvent(hp->d2h, hp->done[c], 0)) ||
             !ok(cudaMemcpyAsync((char*)K_out + rowO * u0, dKo + rowO * u0, rowO * nu, cudaMemcpyDeviceToHost, hp->d2h)) ||
             !ok(cudaMemcpyAsync((char*)V_out + rowO * u0, dVo + rowO * u0, rowO * nu, cudaMemcpyDeviceToHost, hp->d2h)) ||
             !ok(cudaMemcpyAsync(out_len + u0, (int32_t*)dL + u0, (size_t)nu * sizeof(int32_t), cudaMemcpyDeviceToHost,
                                 hp->d2h)) ||
             !ok(cudaMemcpyAsync((char*)out_pos + rowP * u0, dP + rowP * u0, rowP * nu, cudaMemcpyDeviceToHost, hp->d2h)))
-            return KVM_E_CUDA;
+            status = KVM_E_CUDA;
     }
-    if (!ok(cudaEventRecord(hp->end, hp->d2h)) || !ok(cudaStreamWaitEvent(st, hp->end, 0))) return KVM_E_CUDA;
-    return KVM_OK;
+    // join: the copy-out stream follows the compute stream, the caller's stream follows the copy-out stream
+    if (!ok(cudaEventRecord(hp->done[0], hp->compute)) || !ok(cudaStreamWaitEvent(hp->d2h, hp->done[0], 0)) ||
+        !ok(cudaEventRecord(hp->end, hp->d2h)) || !ok(cudaStreamWaitEvent(st, hp->end, 0)))
+        return KVM_E_CUDA;
+    return status;
 }
 
 // ---------------------------------------------------------------------------
@@ -453,13 +478,11 @@ int kvm_compress_host(const kvm_params* p, const void* Q, const void* K, const v
 // The scratch is part of the library image; see the declaration in kvm.h.
 namespace {
 
-constexpr int kMaxDevices = 64;
-constexpr size_t kStaticCounterBytes = 256;
+constexpr int kMaxDevices = KVM_MAX_DEVICES;
 
-// [counters | row log-sum-exp].  In HOST code this name is only a stand-in for
-// the device symbol; its device address comes from cudaGetSymbolAddress below.
-static __device__ __align__(256) unsigned char g_static_score_scratch[kStaticCounterBytes +
-                                                                       (size_t)KVM_STATIC_SCORE_ROWS * sizeof(float)];
+// The row pass's output for up to KVM_STATIC_SCORE_ROWS fp32 rows.  In HOST code this name is only a stand-in
+// for the device symbol; its device address comes from cudaGetSymbolAddress below.
+static __device__ __align__(256) unsigned char g_static_score_scratch[(size_t)KVM_STATIC_SCORE_ROWS * sizeof(float)];
 
 void* g_static_ptr[kMaxDevices];   // device address of the array, per device; set once
 
@@ -488,12 +511,10 @@ int kvm_score_static(const kvm_params* p, const void* Q, const void* K, float* s
     unsigned char* base = (unsigned char*)static_scratch_for_current_device();
     if (!base) return KVM_E_CUDA;
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    // The array keeps the previous call's contents: counters must start at zero; the
-    // log-sum-exp rows are fully rewritten by the row pass before the column pass reads them.
-    if (cudaMemsetAsync(base, 0, kStaticCounterBytes, st) != cudaSuccess) return KVM_E_CUDA;
+    // The array keeps the previous call's contents.  Nothing in it has to start at zero: the row pass rewrites
+    // every row this call's column pass reads.
     Workspace w;
-    w.counters = (int*)base;
-    w.lse = (float*)(base + kStaticCounterBytes);
+    w.lse = (float*)base;
     w.scores = nullptr;
     w.sim = nullptr;
     w.set_start = nullptr;

@@ -8,6 +8,8 @@
 
 namespace kvm {
 
+constexpr int KVM_MAX_DEVICES = 64;   // per-device host-side caches are arrays of this size
+
 // Validated, derived problem sizes handed to every launcher.
 struct Dims {
     int B, Hq, Hkv, G, S, D, U;
@@ -95,7 +97,7 @@ cudaError_t launch_token_sets(const Dims& d, const int32_t* set_start, const int
 cudaError_t launch_merge(const Dims& d, const void* K, const void* V, const int32_t* set_start,
                          const int32_t* pivot, const int32_t* set_id, const int32_t* out_len, void* K_out,
                          void* V_out, int32_t* out_size, float* scratch, float* set_coef, float* token_d2,
-                         cudaStream_t st);
+                         kvm_stats* stats, cudaStream_t st);
 // Rows that are one input state each (pivot-only weights, eviction): a gather.
 cudaError_t launch_gather(const Dims& d, const void* K, const void* V, const int32_t* set_start,
                           const int32_t* pivot, const int32_t* out_len, void* K_out, void* V_out, int32_t* out_size,

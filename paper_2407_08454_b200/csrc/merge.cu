@@ -81,7 +81,8 @@ __global__ void __launch_bounds__(MERGE_NT) merge_tile_kernel(const T* __restric
                                                               T* __restrict__ K_out, T* __restrict__ V_out,
                                                               int32_t* __restrict__ out_size, Slots<D> slots, int S,
                                                               int cap, float neg_inv_2s2_log2e, int scale_v,
-                                                              int average, const float* __restrict__ set_coef) {
+                                                              int average, const float* __restrict__ set_coef,
+                                                              kvm_stats* stats) {
     using Gm = MergeGeom<T, D>;
     constexpr int N = Gm::N, LPR = Gm::LPR, NWORK = Gm::NWORK, NCH = Gm::NCH;
     constexpr int CHL = TOK / NCH;                    // tokens per chunk
@@ -131,11 +132,19 @@ __global__ void __launch_bounds__(MERGE_NT) merge_tile_kernel(const T* __restric
     }
     __syncthreads();                     // barrier initialised + metadata visible
     {
-        // The copies were issued by this block and always complete; the wait is still bounded.
+        // The copies were issued by this block and always complete; the wait is still bounded.  If it ever ran
+        // out, the tile's staged rows are replaced by NaN patterns (so every row this block writes is NaN rather
+        // than whatever shared memory held) and the condition is reported.
         uint32_t done = 0;
         for (uint32_t it = 0; it < (1u << 26) && !done; ++it)
             asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n\t"
                          "selp.u32 %0, 1, 0, p;\n\t}" : "=r"(done) : "r"(smem_u32(&bar)) : "memory");
+        if (!__syncthreads_and((int)done)) {
+            for (int i = threadIdx.x; i < (int)(2 * TOK * D * sizeof(T) / sizeof(uint32_t)); i += MERGE_NT)
+                reinterpret_cast<uint32_t*>(sK)[i] = 0xFFFFFFFFu;
+            if (threadIdx.x == 0 && stats) stats->status = KVM_E_DEVICE_TIMEOUT;
+            __syncthreads();
+        }
     }
 
     const int w = threadIdx.x / LPR, lane = threadIdx.x % LPR;
@@ -399,7 +408,7 @@ cudaError_t launch_gather_t(const Dims& d, const void* K, const void* V, const i
 template <typename T, int D, int TOK>
 cudaError_t launch_t(const Dims& d, const void* K, const void* V, const int32_t* set_start, const int32_t* pivot,
                      const int32_t* set_id, const int32_t* out_len, void* K_out, void* V_out, int32_t* out_size,
-                     float* scratch, float* set_coef, float* token_d2, cudaStream_t st) {
+                     float* scratch, float* set_coef, float* token_d2, kvm_stats* stats, cudaStream_t st) {
     const int Tn = (d.S + TOK - 1) / TOK;
     Slots<D> slots;
     slots.sums = scratch;
@@ -423,7 +432,7 @@ cudaError_t launch_t(const Dims& d, const void* K, const void* V, const int32_t*
     e = launch_dependent(merge_tile_kernel<T, D, TOK>, dim3(Tn, d.U), dim3(MERGE_NT), smem, st, (const T*)K,
                          (const T*)V, set_start, pivot, set_id, (T*)K_out, (T*)V_out, out_size, slots, d.S, d.cap, c,
                          d.scale_v, d.weight_rule == KVM_WEIGHT_AVERAGE ? 1 : 0,
-                         per_set ? (const float*)set_coef : (const float*)nullptr);
+                         per_set ? (const float*)set_coef : (const float*)nullptr, stats);
     if (e != cudaSuccess) return e;
     if (Tn > 1)
         e = launch_dependent(merge_fixup_kernel<T, D, TOK>, dim3(Tn - 1, d.U), dim3(2 * D), 0, st, set_start, set_id,
@@ -467,17 +476,17 @@ cudaError_t launch_gather(const Dims& d, const void* K, const void* V, const int
 cudaError_t launch_merge(const Dims& d, const void* K, const void* V, const int32_t* set_start,
                          const int32_t* pivot, const int32_t* set_id, const int32_t* out_len, void* K_out,
                          void* V_out, int32_t* out_size, float* scratch, float* set_coef, float* token_d2,
-                         cudaStream_t st) {
+                         kvm_stats* stats, cudaStream_t st) {
     if (d.dtype == KVM_BF16) {
         return d.D == 128 ? launch_t<__nv_bfloat16, 128, KVM_MERGE_TOK_BF16>(d, K, V, set_start, pivot, set_id, out_len,
-                                                                          K_out, V_out, out_size, scratch, set_coef, token_d2, st)
+                                                                          K_out, V_out, out_size, scratch, set_coef, token_d2, stats, st)
                           : launch_t<__nv_bfloat16, 64, KVM_MERGE_TOK_BF16>(d, K, V, set_start, pivot, set_id, out_len,
-                                                                         K_out, V_out, out_size, scratch, set_coef, token_d2, st);
+                                                                         K_out, V_out, out_size, scratch, set_coef, token_d2, stats, st);
     }
     return d.D == 128 ? launch_t<float, 128, 64>(d, K, V, set_start, pivot, set_id, out_len, K_out, V_out, out_size,
-                                                 scratch, set_coef, token_d2, st)
+                                                 scratch, set_coef, token_d2, stats, st)
                       : launch_t<float, 64, 64>(d, K, V, set_start, pivot, set_id, out_len, K_out, V_out, out_size,
-                                                scratch, set_coef, token_d2, st);
+                                                scratch, set_coef, token_d2, stats, st);
 }
 
 }  // namespace kvm

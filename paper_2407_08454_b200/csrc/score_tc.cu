@@ -23,7 +23,9 @@
 //
 // One CTA per SM, persistent, warp-specialised:
 //   warps 0-15 epilogue: two groups of 8 take alternate steps; a warp reads TMEM lanes
-//              32*(w%4).. and one column half, does exp2 on the SFUs, keeps row/column state
+//              32*(w%4).. and one column half, does exp2 on the SFUs, keeps row/column state;
+//              steps that no mask touches (all but an item's diagonal and ragged tiles) run
+//              straight-line code, the others a general path
 //   warp  16   producer: TMA (cp.async.bulk.tensor, 128B swizzle) into a 2-stage ring of B pairs
 //   warp  17   MMA issue: one thread issues tcgen05.mma / tcgen05.commit; owns TMEM
 // Work items are dealt in descending length, boustrophedon over the CTAs, which
@@ -34,7 +36,14 @@
 // barriers' payloads, finishes its loops without waiting, the outputs of the
 // affected items are poisoned with NaN, kvm_stats.status is set when given,
 // tensor memory is freed and the kernel returns.
+//
+// Two compile-time switches exist for the test of that give-up path and are never set in the
+// library that ships: KVM_TEST_WAIT_LIMIT_CLOCKS shortens the limit of every wait, and
+// KVM_TEST_DROP_B_STAGE = k makes the producer leave out its k-th B stage (barrier not armed,
+// copies not issued), so that the MMA warp's wait for it runs out.
 #include <cuda.h>
+
+#include <mutex>
 
 #include "similarity_core.cuh"
 
@@ -48,12 +57,17 @@ constexpr int NACC = 2;              // TMEM accumulator ring (2 x 256 columns =
 constexpr int ACC_COLS = 2 * TILE;   // accumulator columns per step
 constexpr int PCH = 16;              // channels of the lse side tensor (one K = 16 MMA slice; 3 are used)
 constexpr uint32_t PTILE_BYTES = TILE * PCH * 2;   // 4 KB: 128 rows x 32 B
-constexpr int NEPI_WARPS = 16;          // 4 TMEM lane quarters x 4 column quarters
-constexpr int QCOLS = TILE / 4;          // accumulator columns per epilogue warp
+constexpr int NEPI_WARPS = 16;           // 4 TMEM lane quarters x 2 groups x 2 column halves
+constexpr int QCOLS = TILE / 4;          // columns of one TMEM load (a "quarter" of a sub-tile)
+constexpr int QPW = 2;                   // quarters of a 128-column sub-tile a warp owns
 constexpr int NSIM_WARPS = 2;           // neighbour-key similarities on the side (one of the two passes)
 constexpr int SIM_RUN = 8;              // consecutive tokens per lane group and round trip
 constexpr int NTHREADS = (NEPI_WARPS + 2 + NSIM_WARPS) * 32;
+#ifdef KVM_TEST_WAIT_LIMIT_CLOCKS
+constexpr long long WAIT_LIMIT_CLOCKS = KVM_TEST_WAIT_LIMIT_CLOCKS;
+#else
 constexpr long long WAIT_LIMIT_CLOCKS = 4000000000ll;   // ~2 s of SM clocks: a longer wait is reported, not endured
+#endif
 constexpr float LOG2E = 1.4426950408889634f;
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -129,18 +143,24 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                  : "memory");
 }
-// 32 consecutive fp32 columns of this thread's TMEM lane, starting at taddr.  The wait is part of the
-// same statement so that no use of the registers can be scheduled before the data has landed.
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
-    uint32_t r[32];
+// 32 consecutive fp32 columns of this thread's TMEM lane, starting at taddr: the load is issued and left in
+// flight.  The registers must not be read before tmem_ld_fence() has been applied to them.
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t* r) {
     asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n\t"
-        "tcgen05.wait::ld.sync.aligned;"
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
         : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr)
         : "memory");
-#pragma unroll
-    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+// Waits for every TMEM load this thread has in flight.
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// Ties 32 loaded registers to the preceding wait: the compiler sees them rewritten here, so no use can be
+// scheduled ahead of the wait.  Emits no instruction.
+__device__ __forceinline__ void tmem_ld_fence(uint32_t* r) {
+    asm volatile(""
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]), "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+                 :
+                 : "memory");
 }
 
 __device__ __forceinline__ float ex2(float x) {
@@ -162,53 +182,10 @@ __device__ __forceinline__ uint64_t ffma2(uint64_t a, uint64_t b, uint64_t c) {
     asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
     return r;
 }
-__device__ __forceinline__ uint64_t fadd2(uint64_t a, uint64_t b) {
-    uint64_t r;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
-}
 __device__ __forceinline__ uint64_t fmul2(uint64_t a, uint64_t b) {
     uint64_t r;
     asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
     return r;
-}
-__device__ __forceinline__ uint64_t fsub2(uint64_t a, uint64_t b) {
-    uint64_t r;
-    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
-}
-// 2^x for a packed pair on the FMA and integer pipes, so that the special-function unit (the
-// bottleneck of both passes: one exponential per logit) only has to serve part of the columns.
-// Textbook scheme: n = round(x) read off the mantissa after adding 1.5*2^23, f = x - n in
-// [-1/2, 1/2], 2^f by a degree-4 minimax polynomial (max relative error 2.7e-6, coefficients fitted
-// for this file), 2^n applied by adding n to the exponent field.  Inputs are clamped at -125, where
-// the result (3e-38) is far below anything that matters in a sum of probabilities.
-__device__ __forceinline__ uint64_t ex2_poly2(uint64_t x2) {
-    float x0, x1;
-    unpack2(x2, x0, x1);
-    const uint64_t xc = pack2(fmaxf(x0, -125.f), fmaxf(x1, -125.f));
-    const uint64_t magic = pack2(12582912.f, 12582912.f);
-    const uint64_t t = fadd2(xc, magic);
-    const uint64_t f = fsub2(xc, fsub2(t, magic));
-    uint64_t p = ffma2(pack2(0.009570102207362652f, 0.009570102207362652f), f,
-                       pack2(0.05591785907745361f, 0.05591785907745361f));
-    p = ffma2(p, f, pack2(0.240247443318367f, 0.240247443318367f));
-    p = ffma2(p, f, pack2(0.6931217908859253f, 0.6931217908859253f));
-    p = ffma2(p, f, pack2(0.9999992847442627f, 0.9999992847442627f));
-    const uint32_t r0 = (uint32_t)p + ((uint32_t)t << 23);
-    const uint32_t r1 = (uint32_t)(p >> 32) + ((uint32_t)(t >> 32) << 23);
-    return ((uint64_t)r1 << 32) | r0;
-}
-// Pair k (of 16) of a 32-column chunk takes the polynomial route when bit k is set.
-#ifndef KVM_POLY_PAIRS
-#define KVM_POLY_PAIRS 0x0u
-#endif
-constexpr uint32_t POLY_PAIRS = KVM_POLY_PAIRS;   // default: none (measured: any share made both passes slower)
-__device__ __forceinline__ uint64_t ex2_pair(uint64_t x2, int k) {
-    if ((POLY_PAIRS >> k) & 1u) return ex2_poly2(x2);
-    float x0, x1;
-    unpack2(x2, x0, x1);
-    return pack2(ex2(x0), ex2(x1));
 }
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
     float r;
@@ -245,6 +222,49 @@ constexpr uint32_t idesc_for(int n) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(TILE >> 4) << 24);
 }
 constexpr uint32_t IDESC_N128 = idesc_for(TILE), IDESC_N256 = idesc_for(2 * TILE);
+
+// ------------------------------------------------------------------ per-chunk arithmetic of the two passes
+// A chunk is 32 consecutive accumulator columns of this thread's row, already masked with -inf where the
+// causal mask or the sequence end excludes them.  The exponentials' results are added one by one: packing them
+// into pairs for a packed add costs a register move per result, which is more than the add it saves.
+//
+// Row pass: fold the chunk into the running maximum m and sum l (log2 units: x = v * scale2).
+__device__ __forceinline__ void chunk_row_pass(const float (&v)[QCOLS], float& m, float& l, float scale2, uint64_t sc2) {
+    float mx[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        mx[c] = fmax3(v[c], v[c + 4], v[c + 8]);
+        mx[c] = fmax3(mx[c], v[c + 12], v[c + 16]);
+        mx[c] = fmax3(mx[c], v[c + 20], v[c + 24]);
+        mx[c] = fmaxf(mx[c], v[c + 28]);
+    }
+    const float mtile = fmaxf(fmax3(mx[0], mx[1], mx[2]), mx[3]);
+    const float mnew = fmaxf(m, mtile * scale2);
+    if (mnew > -INFINITY) {
+        // packed multiply-add for the exponents (the accumulator registers come in adjacent pairs)
+        const uint64_t nm2 = pack2(-mnew, -mnew);
+        float sum[8] = {l * ex2(m - mnew), 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int c = 0; c < QCOLS; c += 2) {
+            float x0, x1;
+            unpack2(ffma2(pack2(v[c], v[c + 1]), sc2, nm2), x0, x1);
+            sum[c & 7] += ex2(x0);
+            sum[(c + 1) & 7] += ex2(x1);
+        }
+        l = ((sum[0] + sum[1]) + (sum[2] + sum[3])) + ((sum[4] + sum[5]) + (sum[6] + sum[7]));
+        m = mnew;
+    }
+}
+// Column pass: the accumulator already holds q.k - lse/c; scale, exponentiate, add to eight partial sums.
+__device__ __forceinline__ void chunk_col_pass(const float (&v)[QCOLS], float (&acc)[8], uint64_t sc2) {
+#pragma unroll
+    for (int c = 0; c < QCOLS; c += 2) {
+        float x0, x1;
+        unpack2(fmul2(pack2(v[c], v[c + 1]), sc2), x0, x1);
+        acc[c & 7] += ex2(x0);
+        acc[(c + 1) & 7] += ex2(x1);
+    }
+}
 
 // ------------------------------------------------------------------ static schedule
 struct Sched {
@@ -301,12 +321,13 @@ struct alignas(16) Shared {
     float part_l[2][3][TILE];
 };
 
-template <int KCH>
+template <int KCH, int PASS>
 __global__ void __launch_bounds__(NTHREADS, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ CUtensorMap map_p, __nv_bfloat16* __restrict__ lsep_out,
-                float* __restrict__ scores, kvm_stats* stats, int pass, int B, int Hq, int Hkv, int S,
+                float* __restrict__ scores, kvm_stats* stats, int B, int Hq, int Hkv, int S,
                 float scale2, const __nv_bfloat16* __restrict__ Ksim, float* __restrict__ sim_out) {
+    constexpr int pass = PASS;
     extern __shared__ uint8_t smem_raw[];
     constexpr uint32_t CHUNK_BYTES = TILE * 128;            // one [128 rows x 64 bf16] TMA box
     constexpr uint32_t TILE_BYTES = KCH * CHUNK_BYTES;      // an A tile: [KCH][128 rows][128 B]
@@ -377,6 +398,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     const int nh = (t + 1 < nt) ? 2 : 1;
                     ok = mbar_wait(&sh.bar.empty_b[s], ((cnt / NSTAGE) & 1) ^ 1, abort_flag);
                     if (!ok) break;
+#ifdef KVM_TEST_DROP_B_STAGE
+                    if (cnt == (uint32_t)(KVM_TEST_DROP_B_STAGE)) continue;   // test build only: this stage never arrives
+#endif
                     last_b[s] = (cnt / NSTAGE) & 1;
                     mbar_expect_tx(&sh.bar.full_b[s], nh * (TILE_BYTES + (pass == 2 ? PTILE_BYTES : 0u)));
                     for (int h = 0; h < nh; ++h) {
@@ -462,21 +486,22 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         }
     } else {
         // ============================== epilogue ==============================
-        // Two groups of 8 warps take alternate steps (group g always reads accumulator stage g), so that
-        // one group's waits, TMEM loads and bookkeeping overlap the other group's exponentials.  Within a
-        // group a warp owns TMEM lane quarter lq and one 64-column half of each 128-column sub-tile,
-        // handled as two 32-column chunks.
+        // Two groups of warps take alternate steps (group g always reads accumulator stage g), so that one
+        // group's waits, TMEM loads and bookkeeping overlap the other group's exponentials.  Within a group a
+        // warp owns TMEM lane quarter lq and QPW 32-column quarters of each 128-column sub-tile, fetched LDQ
+        // quarters at a time; the accumulator is handed back as soon as the step's last fetch has landed.
         const int lq = warp & 3;                             // TMEM lane quarter this warp may read
         const int grp = (warp >> 2) & 1;                     // steps with (cnt & 1) == grp
-        const int chalf = warp >> 3;                         // column half of a sub-tile
-        const int pidx = warp >> 2;                          // partial-sum slot of this warp's row state (0..3)
+        const int part = warp >> 3;                          // which share of a sub-tile's columns (0 when 8 warps)
+        const int pidx = warp >> 2;                          // partial-state slot of this warp's rows
         const int row = lq * 32 + lane;                      // A row = TMEM lane
-        const uint32_t t_lane = tmem_base + ((uint32_t)(lq * 32) << 16) + grp * ACC_COLS + chalf * 64;
+        const uint32_t t_lane = tmem_base + ((uint32_t)(lq * 32) << 16) + grp * ACC_COLS + part * (QPW * QCOLS);
         const uint64_t sc2 = pack2(scale2, scale2);
         bool ok = true;
         StepIter it;
         it.init(sc);
-        uint32_t own = 0;                                    // own steps processed (accumulator phase, staging parity)
+        uint32_t own = 0;                                    // own steps processed (accumulator phase)
+        const bool ragged = (S & (TILE - 1)) != 0;
         while (it.valid) {
             const int n = it.n, head = it.head, tile = it.tile;
             float m = -INFINITY, l = 0.f;                    // pass 1 state
@@ -487,91 +512,92 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 ok = mbar_wait(&sh.bar.acc_full[grp], own & 1, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
                 if (ok) tc_fence_after();
-                int btile = (pass == 1) ? it.t0 : it.bt;
-                for (int h = 0; h < nh; ++h) {
-                    const bool diag = (btile == tile);
+                const int bt0 = (pass == 1) ? it.t0 : it.bt;                        // B tiles of the two sub-tiles
+                const int bt1 = (pass == 1) ? it.t0 + 1 : (it.bt + 1 == T ? tile : it.bt + 1);
+                bool interior = ok && nh == 2 && bt0 != tile && bt1 != tile;
+                if (pass == 2 && ragged) interior = interior && bt0 != T - 1 && bt1 != T - 1;
+                if (interior) {
+                    // no mask anywhere in this step: straight-line code
 #pragma unroll
-                    for (int k = 0; k < 2; ++k) {
-                        const int cq = chalf * 2 + k;            // column quarter of this 32-column chunk
-                        // On the diagonal tile whole quarters are masked (skip) or fully valid (no per-element mask).
-                        const bool skip = diag && ((pass == 1) ? (cq > lq) : (cq < lq));
-                        const bool mask = diag && (cq == lq);
-                        float v[QCOLS];
-                        if (ok && !skip) tmem_ld32(t_lane + h * TILE + k * QCOLS, v);
-                        if (h == nh - 1 && k == 1) {         // last read of this accumulator: release it
+                    for (int ch = 0; ch < 2 * QPW; ++ch) {
+                        uint32_t vr[QCOLS];
+                        tmem_ld32_issue(t_lane + (ch / QPW) * TILE + (ch % QPW) * QCOLS, vr);
+                        tmem_ld_wait();
+                        if (ch == 2 * QPW - 1) {              // last read of this accumulator: release it
                             tc_fence_before();
                             __syncwarp();
                             if (lane == 0) mbar_arrive(&sh.bar.acc_empty[grp]);
                         }
-                        if (!ok || skip) continue;
-                        if (pass == 1) {
-                            if (mask) {
+                        tmem_ld_fence(vr);
+                        float v[QCOLS];
 #pragma unroll
-                                for (int c = 0; c < QCOLS; ++c)
-                                    if (c > lane) v[c] = -INFINITY;      // key after query
+                        for (int c = 0; c < QCOLS; ++c) v[c] = __uint_as_float(vr[c]);
+                        if (pass == 1) chunk_row_pass(v, m, l, scale2, sc2);
+                        else chunk_col_pass(v, acc, sc2);
+                    }
+                } else {
+                    int btile = bt0;
+                    for (int h = 0; h < nh; ++h) {
+                        const bool diag = (btile == tile);
+#pragma unroll 1
+                        for (int k = 0; k < QPW; ++k) {
+                            const int cq = part * QPW + k;       // column quarter of this chunk within the sub-tile
+                            // On the diagonal tile whole quarters are masked (skip) or fully valid.
+                            const bool skip = !ok || (diag && ((pass == 1) ? (cq > lq) : (cq < lq)));
+                            const bool mask = diag && (cq == lq);
+                            uint32_t vr[QCOLS];
+                            if (!skip) { tmem_ld32_issue(t_lane + h * TILE + k * QCOLS, vr); tmem_ld_wait(); }
+                            if (h == nh - 1 && k == QPW - 1) {
+                                tc_fence_before();
+                                __syncwarp();
+                                if (lane == 0) mbar_arrive(&sh.bar.acc_empty[grp]);
                             }
-                            float mx[4];
+                            if (skip) continue;
+                            tmem_ld_fence(vr);
+                            float v[QCOLS];
 #pragma unroll
-                            for (int c = 0; c < 4; ++c) {
-                                mx[c] = fmax3(v[c], v[c + 4], v[c + 8]);
-                                mx[c] = fmax3(mx[c], v[c + 12], v[c + 16]);
-                                mx[c] = fmax3(mx[c], v[c + 20], v[c + 24]);
-                                mx[c] = fmaxf(mx[c], v[c + 28]);
-                            }
-                            const float mtile = fmaxf(fmax3(mx[0], mx[1], mx[2]), mx[3]);
-                            const float mnew = fmaxf(m, mtile * scale2);
-                            if (mnew > -INFINITY) {
-                                const uint64_t nm2 = pack2(-mnew, -mnew);
-                                // packed multiply-add for the exponents (the accumulator registers come in
-                                // adjacent pairs); the exponentials are summed in eight scalar chains
-                                float sum[8] = {l * ex2(m - mnew), 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                            for (int c = 0; c < QCOLS; ++c) v[c] = __uint_as_float(vr[c]);
+                            if (pass == 1) {
+                                if (mask) {
 #pragma unroll
-                                for (int c = 0; c < QCOLS; c += 2) {
-                                    float e0, e1;
-                                    unpack2(ex2_pair(ffma2(pack2(v[c], v[c + 1]), sc2, nm2), c >> 1), e0, e1);
-                                    sum[c & 7] += e0;
-                                    sum[(c + 1) & 7] += e1;
+                                    for (int c = 0; c < QCOLS; ++c)
+                                        if (c > lane) v[c] = -INFINITY;      // key after query
                                 }
-                                l = ((sum[0] + sum[1]) + (sum[2] + sum[3])) + ((sum[4] + sum[5]) + (sum[6] + sum[7]));
-                                m = mnew;
-                            }
-                        } else {
-                            // The accumulator already holds q.k - lse/c: mask, scale, exponentiate, add.
-                            const int ncol = S - btile * TILE - cq * QCOLS;   // live columns of this chunk (queries < S)
-                            if (mask || ncol < QCOLS) {
+                                chunk_row_pass(v, m, l, scale2, sc2);
+                            } else {
+                                const int ncol = S - btile * TILE - cq * QCOLS;   // live columns of this chunk (queries < S)
+                                if (mask || ncol < QCOLS) {
 #pragma unroll
-                                for (int c = 0; c < QCOLS; ++c)
-                                    if ((mask && c < lane) || c >= ncol) v[c] = -INFINITY;   // query before key, or past the end
-                            }
-#pragma unroll
-                            for (int c = 0; c < QCOLS; c += 2) {
-                                float e0, e1;
-                                unpack2(ex2_pair(fmul2(pack2(v[c], v[c + 1]), sc2), c >> 1), e0, e1);
-                                acc[c & 7] += e0;
-                                acc[(c + 1) & 7] += e1;
+                                    for (int c = 0; c < QCOLS; ++c)
+                                        if ((mask && c < lane) || c >= ncol) v[c] = -INFINITY;   // query before key, or past the end
+                                }
+                                chunk_col_pass(v, acc, sc2);
                             }
                         }
+                        btile = bt1;
                     }
-                    if (++btile == T && pass == 2) btile = tile;
                 }
                 ++own;
             }
             // ---- item end: combine the four partial states of every row (fixed order) and store
-            const bool bad = (*abort_flag != 0);
             const int slot = n & 1;
             const float mine = (pass == 1) ? l : ((acc[0] + acc[1]) + (acc[2] + acc[3])) + ((acc[4] + acc[5]) + (acc[6] + acc[7]));
+            constexpr int NPART = NEPI_WARPS / 4;            // partial states per row (one per warp that owns it)
             if (pidx > 0) { sh.part_m[slot][pidx - 1][row] = m; sh.part_l[slot][pidx - 1][row] = mine; }
             named_bar(5, NEPI_WARPS * 32);
+            // (read after the barrier: a warp that had no step left when another warp's wait ran out must still
+            // see the flag, or it would store sums that lack the abandoned steps)
+            const bool bad = (*abort_flag != 0);
             if (pidx == 0) {
                 const int gi = tile * TILE + row;
                 if (gi < S) {
                     if (pass == 1) {
                         float M = m;
 #pragma unroll
-                        for (int q = 0; q < 3; ++q) M = fmaxf(M, sh.part_m[slot][q][row]);
+                        for (int q = 0; q < NPART - 1; ++q) M = fmaxf(M, sh.part_m[slot][q][row]);
                         float L = (m > -INFINITY) ? l * ex2(m - M) : 0.f;
 #pragma unroll
-                        for (int q = 0; q < 3; ++q) {
+                        for (int q = 0; q < NPART - 1; ++q) {
                             const float mq = sh.part_m[slot][q][row], lq_ = sh.part_l[slot][q][row];
                             if (mq > -INFINITY) L += lq_ * ex2(mq - M);
                         }
@@ -586,7 +612,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                                             (uint32_t)__bfloat16_as_ushort(el), 0u, 0u);
                         dst[1] = make_uint4(0u, 0u, 0u, 0u);
                     } else {
-                        const float tot = (mine + sh.part_l[slot][0][row]) + (sh.part_l[slot][1][row] + sh.part_l[slot][2][row]);
+                        float tot = mine;
+#pragma unroll
+                        for (int q = 0; q < NPART - 1; ++q) tot += sh.part_l[slot][q][row];
                         scores[(size_t)head * S + gi] = bad ? NAN : tot / (float)G;
                     }
                 }
@@ -678,19 +706,33 @@ cudaError_t launch_t(const Dims& d, const CUtensorMap& mq, const CUtensorMap& mk
                      const __nv_bfloat16* Ksim, float* sim_out, float* lse_out) {
     const size_t smem = 1024 + (size_t)(2 + 2 * NSTAGE) * KCH * TILE * 128 + (size_t)(2 * NSTAGE + 1) * PTILE_BYTES +
                         sizeof(Shared);
-    cudaError_t e = cudaFuncSetAttribute(score_tc_kernel<KCH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
+    // the shared-memory opt-in and the SM count are looked up once per device and kernel instantiation
+    static std::mutex mu;
+    static int sms_of[KVM_MAX_DEVICES] = {};
+    cudaError_t e;
     int dev = 0, sms = 0;
     if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
-    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+    if (dev < 0 || dev >= KVM_MAX_DEVICES) return cudaErrorInvalidDevice;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        if (!sms_of[dev]) {
+            e = cudaFuncSetAttribute(score_tc_kernel<KCH, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+            e = cudaFuncSetAttribute(score_tc_kernel<KCH, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+            if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+            sms_of[dev] = sms;
+        }
+        sms = sms_of[dev];
+    }
     const int T = (d.S + TILE - 1) / TILE;
     const float scale2 = d.scale * LOG2E;
     if (!lse_in) {
         const long long items = (long long)d.B * d.Hq * T;
         const int grid = (int)(items < sms ? items : sms);
         // (the kernel begins with the dependency wait, so it may be scheduled while whatever precedes it drains)
-        e = launch_dependent(score_tc_kernel<KCH>, dim3(grid), dim3(NTHREADS), smem, st, mq, mk, mp, side,
-                             (float*)nullptr, stats, 1, d.B, d.Hq, d.Hkv, d.S, scale2, Ksim, sim_out);
+        e = launch_dependent(score_tc_kernel<KCH, 1>, dim3(grid), dim3(NTHREADS), smem, st, mq, mk, mp, side,
+                             (float*)nullptr, stats, d.B, d.Hq, d.Hkv, d.S, scale2, Ksim, sim_out);
         if (e != cudaSuccess) return e;
     } else {
         const long long rows = (long long)d.B * d.Hq * d.S;
@@ -707,8 +749,8 @@ cudaError_t launch_t(const Dims& d, const CUtensorMap& mq, const CUtensorMap& mk
     if (!scores) return cudaSuccess;                  // row pass only
     const long long items = (long long)d.U * T;
     const int grid = (int)(items < sms ? items : sms);
-    return launch_dependent(score_tc_kernel<KCH>, dim3(grid), dim3(NTHREADS), smem, st, mq, mk, mp,
-                            (__nv_bfloat16*)nullptr, scores, stats, 2, d.B, d.Hq, d.Hkv, d.S, scale2, Ksim,
+    return launch_dependent(score_tc_kernel<KCH, 2>, dim3(grid), dim3(NTHREADS), smem, st, mq, mk, mp,
+                            (__nv_bfloat16*)nullptr, scores, stats, d.B, d.Hq, d.Hkv, d.S, scale2, Ksim,
                             sim_in_pass2 ? sim_out : (float*)nullptr);
 }
 

@@ -7,15 +7,14 @@ import re
 import pytest
 
 import paper_2407_08454_b200 as kvm
-from paper_2407_08454_b200 import binding, build
+from paper_2407_08454_b200 import binding
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 @pytest.fixture(scope="module")
-def lib():
-    build.build()
-    return binding.lib()
+def lib(kvm_lib):
+    return kvm_lib
 
 
 def test_every_declared_symbol_is_exported(lib):

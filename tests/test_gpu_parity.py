@@ -219,6 +219,7 @@ def test_compress_is_reproducible_bit_for_bit():
     (2, 6, 3, 700, 128, torch.bfloat16),      # 6 units: one per group
     (5, 4, 2, 300, 128, torch.bfloat16),      # 10 units: groups of 2, GQA
     (1, 2, 1, 256, 64, torch.bfloat16),       # a single unit
+    (3, 3, 3, 1001, 64, torch.bfloat16),      # 9 units in groups of 2: a group's pivot keys start 4004 bytes apart
 ])
 def test_host_entry_point_equals_the_device_path(B, Hq, Hkv, S, D, dtype):
     cfg = si.CONFIGS["C1"].scaled(seq=S, head_dim=D, n_q_heads=Hq, n_kv_heads=Hkv, batch=B,
