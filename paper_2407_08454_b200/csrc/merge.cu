@@ -6,18 +6,19 @@
 //
 // Bandwidth-bound, and sets can be arbitrarily long, so the work is split by
 // TOKENS, not by sets: a block owns TOK consecutive tokens of one unit, pulls
-// their K and V rows into shared memory with two bulk copies, and
-//   phase 1  one lane group per token computes its weight g_j (the pivot row is
-//            taken from shared memory when it lies in the tile, else from L2);
-//   phase 2  the tile is cut into short chunks of consecutive tokens; one lane
-//            group per (chunk, tensor) walks its chunk in order with 16-byte
-//            shared-memory reads, adding g_j x_j, and flushes at set boundaries;
-//   phase 3  sets that cross chunk boundaries are completed from per-chunk
-//            "head"/"tail" partial sums kept in shared memory.
-// A set that lies inside the tile is finished there.  A set that crosses tile
-// boundaries leaves fp32 partial sums in a scratch slot per (unit, tile): "head"
-// = the tile's tokens before its first boundary, "tail" = after its last; a small
-// second kernel adds a crossing set's slots in tile order and stores the row.
+// their K and V rows into shared memory with two bulk copies (issued before the
+// kernel even waits for the set data, which comes from the kernel before it), and
+//   weights   one lane group per token computes g_j (the pivot row is taken from
+//             shared memory when it lies in the tile, else from L2);
+//   segments  the tile is cut where the set changes; at most TOK pieces;
+//   walk      a lane group as wide as a K row and a V row together takes every fourth
+//             piece: a piece that is a whole set of one token is copied, a piece that
+//             is a whole set is summed (a loop of 16-byte shared-memory reads and
+//             multiply-adds with no branch in it), scaled and stored; a piece of a set that reaches
+//             beyond the tile leaves its fp32 sums in a scratch slot per (unit, tile):
+//             "head" = the tile's tokens before its first boundary, "tail" = after its
+//             last.  A small second kernel adds a crossing set's slots in tile order and
+//             stores the row.
 // Nothing uses atomics: every sum has a fixed order, results are reproducible.
 // Sets of one token are copied bit for bit.
 // Variants: average-weighted merging (Section 4.2) is the same kernel with every
@@ -63,40 +64,30 @@ template <int D> struct Slots {
     }
 };
 
-constexpr int MERGE_NT = 256;
-
-// Shared-memory footprint of the per-chunk partial sums (see merge_tile_kernel).
-template <typename T, int D> struct MergeGeom {
-    static constexpr int N = Vec<T>::N;              // elements per 16 bytes
-    static constexpr int LPR = D / N;                // lanes per row
-    static constexpr int NWORK = MERGE_NT / LPR;     // lane groups per block
-    static constexpr int NCH = NWORK / 2;            // token chunks per tile (one group per chunk and tensor)
-};
+// Piece kinds of the walk.
+enum : int { PIECE_COPY = 0, PIECE_WHOLE = 1, PIECE_HEAD = 2, PIECE_TAIL = 3 };
 
 template <typename T, int D, int TOK>
-__global__ void __launch_bounds__(MERGE_NT) merge_tile_kernel(const T* __restrict__ K, const T* __restrict__ V,
-                                                              const int32_t* __restrict__ set_start,
-                                                              const int32_t* __restrict__ pivot,
-                                                              const int32_t* __restrict__ set_id,
-                                                              T* __restrict__ K_out, T* __restrict__ V_out,
-                                                              int32_t* __restrict__ out_size, Slots<D> slots, int S,
-                                                              int cap, float neg_inv_2s2_log2e, int scale_v,
-                                                              int average, const float* __restrict__ set_coef,
-                                                              kvm_stats* stats) {
-    using Gm = MergeGeom<T, D>;
-    constexpr int N = Gm::N, LPR = Gm::LPR, NWORK = Gm::NWORK, NCH = Gm::NCH;
-    constexpr int CHL = TOK / NCH;                    // tokens per chunk
-    static_assert(TOK % NCH == 0 && CHL >= 1, "tile must split evenly into chunks");
+__global__ void __launch_bounds__(2 * D) merge_tile_kernel(const T* __restrict__ K, const T* __restrict__ V,
+                                                           const int32_t* __restrict__ set_start,
+                                                           const int32_t* __restrict__ pivot,
+                                                           const int32_t* __restrict__ set_id,
+                                                           T* __restrict__ K_out, T* __restrict__ V_out,
+                                                           int32_t* __restrict__ out_size, Slots<D> slots, int S,
+                                                           int cap, float neg_inv_2s2_log2e, int scale_v, int average,
+                                                           const float* __restrict__ set_coef, kvm_stats* stats) {
+    constexpr int NT = 2 * D;
+    constexpr int N = Vec<T>::N, LPR = D / N, NG = NT / LPR;
+    static_assert(TOK <= 64 && TOK <= NT, "one thread per token for the set data, two ballots for the pieces");
     extern __shared__ __align__(128) uint8_t smem_raw[];
     T* sK = reinterpret_cast<T*>(smem_raw);
     T* sV = sK + TOK * D;
-    // per-chunk partial sums: [chunk][head|tail][K|V][D]
-    float* sPart = reinterpret_cast<float*>(sV + TOK * D);
     __shared__ __align__(8) uint64_t bar;
-    __shared__ int s_sid[TOK], s_piv[TOK], s_beg[TOK], s_end[TOK];
+    __shared__ int s_sid[TOK], s_piv[TOK], s_len[TOK];
     __shared__ float s_g[TOK];
     __shared__ float s_coef[TOK];       // squared distance -> exponent of 2, per token (fixed sigma or the set's own)
-    __shared__ float s_gpart[NCH][2];
+    __shared__ int s_pbeg[TOK + 1], s_pkind[TOK], s_prow[TOK], s_pn[TOK];   // pieces: first token, kind, output row, set size
+    __shared__ int s_npiece, s_warpcnt[2];
 
     const int tile = blockIdx.x, Tn = gridDim.x;
     const long long u = blockIdx.y;
@@ -120,165 +111,143 @@ __global__ void __launch_bounds__(MERGE_NT) merge_tile_kernel(const T* __restric
     }
     // The K and V rows are inputs; everything read from here on comes from the kernel before this one.
     grid_dependency_wait();
-    // per-token set data while the rows are in flight
-    for (int j = threadIdx.x; j < ntok; j += MERGE_NT) {
-        // written by the previous kernel while this block may already have been resident: read through L2
-        const int sid = __ldcg(set_id + (size_t)u * S + tok0 + j);
-        s_sid[j] = sid;
-        s_piv[j] = __ldcg(pivot + (size_t)u * cap + sid);
-        s_beg[j] = __ldcg(st + sid);
-        s_end[j] = __ldcg(st + sid + 1);
-        s_coef[j] = set_coef ? __ldcg(set_coef + (size_t)u * cap + sid) : neg_inv_2s2_log2e;
-    }
-    __syncthreads();                     // barrier initialised + metadata visible
     {
-        // The copies were issued by this block and always complete; the wait is still bounded.  If it ever ran
-        // out, the tile's staged rows are replaced by NaN patterns (so every row this block writes is NaN rather
-        // than whatever shared memory held) and the condition is reported.
-        uint32_t done = 0;
-        for (uint32_t it = 0; it < (1u << 26) && !done; ++it)
-            asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n\t"
-                         "selp.u32 %0, 1, 0, p;\n\t}" : "=r"(done) : "r"(smem_u32(&bar)) : "memory");
-        if (!__syncthreads_and((int)done)) {
-            for (int i = threadIdx.x; i < (int)(2 * TOK * D * sizeof(T) / sizeof(uint32_t)); i += MERGE_NT)
-                reinterpret_cast<uint32_t*>(sK)[i] = 0xFFFFFFFFu;
-            if (threadIdx.x == 0 && stats) stats->status = KVM_E_DEVICE_TIMEOUT;
-            __syncthreads();
-        }
-    }
-
-    const int w = threadIdx.x / LPR, lane = threadIdx.x % LPR;
-    const unsigned gmask = (LPR == 32) ? 0xffffffffu : (((1u << LPR) - 1u) << ((threadIdx.x % 32) / LPR * LPR));
-
-    // ---- phase 1: weights, one lane group per token
-    for (int j = w; j < ntok; j += NWORK) {
-        if (s_end[j] - s_beg[j] == 1) continue;      // a set of one token is copied, its weight is never used
-        const int p = s_piv[j];
-        float kj[N], kp[N];
-        Vec<T>::unpack(*reinterpret_cast<const uint4*>(sK + (size_t)j * D + lane * N), kj);
-        if (p >= tok0 && p < tile_end)
-            Vec<T>::unpack(*reinterpret_cast<const uint4*>(sK + (size_t)(p - tok0) * D + lane * N), kp);
-        else
-            Vec<T>::unpack(ldg16(Ku + (size_t)p * D + lane * N), kp);
-        float d2 = 0.f;
-#pragma unroll
-        for (int e = 0; e < N; ++e) { const float a = kp[e] - kj[e]; d2 = fmaf(a, a, d2); }
-#pragma unroll
-        for (int off = 1; off < LPR; off <<= 1) d2 += __shfl_xor_sync(gmask, d2, off);
-        if (lane == 0) s_g[j] = average ? 1.f : exp2f(d2 * s_coef[j]);
-    }
-    __syncthreads();
-
-    // ---- phase 2: lane group (chunk q, tensor) walks CHL consecutive tokens; a lane owns N channels
-    const int q = w >> 1, which = w & 1;                 // 0: K, 1: V
-    const T* sX = which ? sV : sK;
-    T* out = which ? V_out : K_out;
-    float* partH = sPart + ((size_t)(q * 2 + 0) * 2 + which) * D + lane * N;
-    float* partL = sPart + ((size_t)(q * 2 + 1) * 2 + which) * D + lane * N;
-    const int c0 = q * CHL, c1 = min(c0 + CHL, ntok);     // chunk = tile tokens [c0, c1)
-    if (c0 < ntok) {
-        float acc[N], gs = 0.f;
-#pragma unroll
-        for (int e = 0; e < N; ++e) acc[e] = 0.f;
-        uint4 first_raw = *reinterpret_cast<const uint4*>(sX + (size_t)c0 * D + lane * N);
-        auto flush = [&](int j_last) {   // the set whose last token in this chunk is j_last (tile-relative)
-            const int sid = s_sid[j_last], beg = s_beg[j_last], end = s_end[j_last];
-            const bool started_here = beg >= tok0 + c0, closes_here = end <= tok0 + c1;
-            if (started_here && closes_here) {
-                const int n = end - beg;
-                uint4 r = first_raw;
-                if (n > 1) {
-                    const float mul = (which && scale_v) ? (float)n / gs : 1.f / gs;
-                    float o[N];
-#pragma unroll
-                    for (int e = 0; e < N; ++e) o[e] = acc[e] * mul;
-                    r = Vec<T>::pack(o);
-                }
-                *reinterpret_cast<uint4*>(out + ((size_t)u * cap + sid) * D + lane * N) = r;
-                if (out_size && which == 0 && lane == 0) out_size[(size_t)u * cap + sid] = n;
-            } else {
-                float* dst = started_here ? partL : partH;
-#pragma unroll
-                for (int e = 0; e < N; ++e) dst[e] = acc[e];
-                if (which == 0 && lane == 0) s_gpart[q][started_here ? 1 : 0] = gs;
+        // ---- set data per token and the pieces of the tile, while the rows are in flight
+        {
+            const int j = threadIdx.x;
+            int sid = -1, beg = 0, end = 0;
+            if (j < ntok) {
+                // written by the previous kernel while this block may already have been resident: read through L2
+                sid = __ldcg(set_id + (size_t)u * S + tok0 + j);
+                beg = __ldcg(st + sid);
+                end = __ldcg(st + sid + 1);
+                s_sid[j] = sid;
+                s_len[j] = end - beg;
+                s_piv[j] = __ldcg(pivot + (size_t)u * cap + sid);
+                s_coef[j] = set_coef ? __ldcg(set_coef + (size_t)u * cap + sid) : neg_inv_2s2_log2e;
             }
-        };
-        for (int j = c0; j < c1; ++j) {
-            const uint4 raw = *reinterpret_cast<const uint4*>(sX + (size_t)j * D + lane * N);
-            if (j > c0 && s_sid[j] != s_sid[j - 1]) {
-                flush(j - 1);
+            if (j < 64) {                                     // warps 0 and 1: a piece starts where the set changes
+                const int prev = __shfl_up_sync(0xffffffffu, sid, 1);
+                const bool lane0 = (j & 31) == 0;
+                // (lane 0 of warp 1 compares with token 31, fetched again: the shuffle does not cross warps)
+                const int before = lane0 ? ((j == 0 || j >= ntok) ? -2 : __ldcg(set_id + (size_t)u * S + tok0 + j - 1)) : prev;
+                const bool start = j < ntok && sid != before;
+                const unsigned m = __ballot_sync(0xffffffffu, start);
+                if (lane0) s_warpcnt[j >> 5] = __popc(m);
+                const int below = __popc(m & ((1u << (j & 31)) - 1u));
+                asm volatile("bar.sync 1, 64;" ::: "memory");   // the two warps exchange their counts
+                const int idx = below + ((j >> 5) ? s_warpcnt[0] : 0);
+                if (start) {
+                    int kind;
+                    if (end - beg == 1) kind = PIECE_COPY;
+                    else if (beg >= tok0 && end <= tile_end) kind = PIECE_WHOLE;
+                    else kind = (beg < tok0) ? PIECE_HEAD : PIECE_TAIL;
+                    s_pbeg[idx] = j; s_pkind[idx] = kind; s_prow[idx] = sid; s_pn[idx] = end - beg;
+                }
+                if (j == 0) {
+                    const int np = s_warpcnt[0] + s_warpcnt[1];
+                    s_npiece = np;
+                    s_pbeg[np] = ntok;
+                }
+            }
+        }
+        {
+            // The copies were issued by this block and always complete; the wait is still bounded.  If it ever ran
+            // out, the tile's staged rows are replaced by NaN patterns (so every row this block writes is NaN rather
+            // than whatever shared memory held) and the condition is reported.
+            uint32_t done = 1;
+            if (threadIdx.x == 0) {                      // one thread polls, sparsely; the others wait at the block barrier
+                done = 0;
+                for (uint32_t k = 0; k < (1u << 24) && !done; ++k) {
+                    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n\t"
+                                 "selp.u32 %0, 1, 0, p;\n\t}" : "=r"(done) : "r"(smem_u32(&bar)) : "memory");
+                    if (!done) __nanosleep(100);
+                }
+            }
+            if (!__syncthreads_and((int)done)) {         // (also: set data and pieces visible)
+                for (int i = threadIdx.x; i < (int)(2 * TOK * D * sizeof(T) / sizeof(uint32_t)); i += NT)
+                    reinterpret_cast<uint32_t*>(sK)[i] = 0xFFFFFFFFu;
+                if (threadIdx.x == 0 && stats) stats->status = KVM_E_DEVICE_TIMEOUT;
+                __syncthreads();
+            }
+        }
+
+        // ---- weights, one lane group per token
+        if (!average) {
+            const int w = threadIdx.x / LPR, lane = threadIdx.x % LPR;
+            const unsigned gmask = (LPR == 32) ? 0xffffffffu : (((1u << LPR) - 1u) << ((threadIdx.x % 32) / LPR * LPR));
+#pragma unroll 2
+            for (int j = w; j < ntok; j += NG) {
+                if (s_len[j] == 1) continue;             // a set of one token is copied, its weight is never used
+                const int p = s_piv[j];
+                float kj[N], kp[N];
+                const uint4* sK4 = reinterpret_cast<const uint4*>(sK) + lane;      // rows of LPR 16-byte pieces
+                Vec<T>::unpack(sK4[j * LPR], kj);
+                if (p >= tok0 && p < tile_end)
+                    Vec<T>::unpack(sK4[(p - tok0) * LPR], kp);
+                else
+                    Vec<T>::unpack(ldg16(Ku + (size_t)p * D + lane * N), kp);
+                float d2 = 0.f;
+#pragma unroll
+                for (int e = 0; e < N; ++e) { const float a = kp[e] - kj[e]; d2 = fmaf(a, a, d2); }
+#pragma unroll
+                for (int off = 1; off < LPR; off <<= 1) d2 += __shfl_xor_sync(gmask, d2, off);
+                if (lane == 0) s_g[j] = exp2f(d2 * s_coef[j]);
+            }
+        } else {
+            for (int j = threadIdx.x; j < ntok; j += NT) s_g[j] = 1.f;
+        }
+        __syncthreads();
+
+        // ---- walk: a lane group as wide as a K row and a V row together (a warp at most; then K first, V second)
+        // takes every NWK-th piece; a lane owns 16 bytes of a row
+        constexpr int GL = (2 * LPR <= 32) ? 2 * LPR : 32;   // lanes per walking group
+        constexpr int TPASS = 2 * LPR / GL;                  // tensors handled one after the other (1: side by side)
+        constexpr int NWK = NT / GL;
+        const int wk = threadIdx.x / GL, gl = threadIdx.x % GL;
+        const int np = s_npiece;
+#pragma unroll
+        for (int tp = 0; tp < TPASS; ++tp) {
+            const int which = (TPASS == 2) ? tp : gl / LPR;
+            const int ch = (gl % LPR) * N;
+            const uint4* sX4 = reinterpret_cast<const uint4*>(which ? sV : sK) + (gl % LPR);   // rows of LPR 16-byte pieces
+            uint4* out4 = reinterpret_cast<uint4*>((which ? V_out : K_out) + (size_t)u * cap * D) + (gl % LPR);
+            for (int k = wk; k < np; k += NWK) {
+                const int a = s_pbeg[k], b = s_pbeg[k + 1], kind = s_pkind[k], row = s_prow[k];
+                if (kind == PIECE_COPY) {
+                    out4[row * LPR] = sX4[a * LPR];
+                    if (out_size && gl == 0 && tp == 0) out_size[(size_t)u * cap + row] = 1;
+                    continue;
+                }
+                float acc[N], gs = 0.f;
 #pragma unroll
                 for (int e = 0; e < N; ++e) acc[e] = 0.f;
-                gs = 0.f;
-                first_raw = raw;
-            }
-            if (s_end[j] - s_beg[j] == 1) continue;      // copied from first_raw at its flush
-            const float g = s_g[j];
-            float x[N];
-            Vec<T>::unpack(raw, x);
+                const uint4* px = sX4 + a * LPR;
+                const float* pg = s_g + a;
+#pragma unroll 4
+                for (int n_left = b - a; n_left > 0; --n_left, px += LPR, ++pg) {
+                    const float g = *pg;
+                    float x[N];
+                    Vec<T>::unpack(*px, x);
 #pragma unroll
-            for (int e = 0; e < N; ++e) acc[e] = fmaf(g, x[e], acc[e]);
-            gs += g;
-        }
-        flush(c1 - 1);
-    }
-    __syncthreads();
-
-    // ---- phase 3: sets that cross chunk boundaries.  Boundary q (the start of chunk q; q = 0 is the
-    // tile start) is handled by the same lane group: if a set crosses it and does not cross the next
-    // one, its pieces (tail of the chunk where it began, heads of the chunks it covers) are added in
-    // chunk order and stored as the finished row, or as this tile's head / tail slot when the set
-    // extends beyond the tile.
-    if (c0 < ntok) {
-        const int beg = s_beg[c0], end = s_end[c0], sid = s_sid[c0];
-        const int tokb = tok0 + c0;
-        const bool crosses = beg < tokb;
-        const bool last_in_tile = (tok0 + c1 == tile_end);
-        if (crosses && (end <= tok0 + c1 || last_in_tile)) {
-            float sum[N], gs = 0.f;
+                    for (int e = 0; e < N; ++e) acc[e] = fmaf(g, x[e], acc[e]);
+                    gs += g;
+                }
+                if (kind == PIECE_WHOLE) {
+                    const int n = s_pn[k];
+                    const float mul = (which && scale_v) ? (float)n / gs : 1.f / gs;
 #pragma unroll
-            for (int e = 0; e < N; ++e) sum[e] = 0.f;
-            int qa = 0;
-            if (beg >= tok0) {                               // began in this tile: its chunk holds a tail piece
-                qa = (beg - tok0) / CHL;
-                const float* pl = sPart + ((size_t)(qa * 2 + 1) * 2 + which) * D + lane * N;
+                    for (int e = 0; e < N; ++e) acc[e] *= mul;
+                    out4[row * LPR] = Vec<T>::pack(acc);
+                    if (out_size && gl == 0 && tp == 0) out_size[(size_t)u * cap + row] = n;
+                } else {
+                    const int slot = (kind == PIECE_TAIL) ? 1 : 0;
+                    float* dst = slots.s(u, Tn, tile, slot) + which * D + ch;
 #pragma unroll
-                for (int e = 0; e < N; ++e) sum[e] = pl[e];
-                gs = s_gpart[qa][1];
-                ++qa;
-            }
-            for (int c = qa; c <= q; ++c) {
-                const float* ph = sPart + ((size_t)(c * 2 + 0) * 2 + which) * D + lane * N;
-#pragma unroll
-                for (int e = 0; e < N; ++e) sum[e] += ph[e];
-                gs += s_gpart[c][0];
-            }
-            if (beg >= tok0 && end <= tile_end) {            // whole set inside the tile: finished row
-                const int n = end - beg;
-                const float mul = (which && scale_v) ? (float)n / gs : 1.f / gs;
-                float o[N];
-#pragma unroll
-                for (int e = 0; e < N; ++e) o[e] = sum[e] * mul;
-                *reinterpret_cast<uint4*>(out + ((size_t)u * cap + sid) * D + lane * N) = Vec<T>::pack(o);
-                if (out_size && which == 0 && lane == 0) out_size[(size_t)u * cap + sid] = n;
-            } else {
-                const int slot = (beg >= tok0) ? 1 : 0;      // tail : head of this tile
-                float* dst = slots.s(u, Tn, tile, slot) + which * D + lane * N;
-#pragma unroll
-                for (int e = 0; e < N; ++e) dst[e] = sum[e];
-                if (which == 0 && lane == 0) *slots.g(u, Tn, tile, slot) = gs;
-            }
-        }
-        // a set that begins inside the tile's last chunk and runs past the tile: its tail piece is the tile's tail
-        if (last_in_tile) {
-            const int jl = c1 - 1;
-            const int bl = s_beg[jl], el = s_end[jl];
-            if (bl >= tokb && el > tile_end) {
-                const float* pl = sPart + ((size_t)(q * 2 + 1) * 2 + which) * D + lane * N;
-                float* dst = slots.s(u, Tn, tile, 1) + which * D + lane * N;
-#pragma unroll
-                for (int e = 0; e < N; ++e) dst[e] = pl[e];
-                if (which == 0 && lane == 0) *slots.g(u, Tn, tile, 1) = s_gpart[q][1];
+                    for (int e = 0; e < N; e += 4)
+                        *reinterpret_cast<float4*>(dst + e) = make_float4(acc[e], acc[e + 1], acc[e + 2], acc[e + 3]);
+                    if (gl == 0 && tp == 0) *slots.g(u, Tn, tile, slot) = gs;
+                }
             }
         }
     }
@@ -413,10 +382,8 @@ cudaError_t launch_t(const Dims& d, const void* K, const void* V, const int32_t*
     Slots<D> slots;
     slots.sums = scratch;
     slots.gsum = scratch + (size_t)d.U * Tn * 2 * (2 * D);
-    const size_t smem = (size_t)2 * TOK * D * sizeof(T) + (size_t)MergeGeom<T, D>::NCH * 2 * 2 * D * sizeof(float);
-    cudaError_t e = cudaFuncSetAttribute(merge_tile_kernel<T, D, TOK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)smem);
-    if (e != cudaSuccess) return e;
+    const size_t smem = (size_t)2 * TOK * D * sizeof(T);       // 32 KB: below the default limit, no opt-in needed
+    cudaError_t e = cudaSuccess;
     const float c = -LOG2E / (2.f * d.sigma * d.sigma);
     const bool per_set = d.weight_rule == KVM_WEIGHT_SET_SIGMA;
     if (per_set) {
@@ -429,7 +396,7 @@ cudaError_t launch_t(const Dims& d, const void* K, const void* V, const int32_t*
                              set_start, out_len, set_coef, d.S, d.cap);
         if (e != cudaSuccess) return e;
     }
-    e = launch_dependent(merge_tile_kernel<T, D, TOK>, dim3(Tn, d.U), dim3(MERGE_NT), smem, st, (const T*)K,
+    e = launch_dependent(merge_tile_kernel<T, D, TOK>, dim3(Tn, d.U), dim3(2 * D), smem, st, (const T*)K,
                          (const T*)V, set_start, pivot, set_id, (T*)K_out, (T*)V_out, out_size, slots, d.S, d.cap, c,
                          d.scale_v, d.weight_rule == KVM_WEIGHT_AVERAGE ? 1 : 0,
                          per_set ? (const float*)set_coef : (const float*)nullptr, stats);
@@ -446,7 +413,7 @@ cudaError_t launch_t(const Dims& d, const void* K, const void* V, const int32_t*
 #ifndef KVM_MERGE_TOK_BF16
 #define KVM_MERGE_TOK_BF16 64
 #endif
-static int merge_tile_tokens(const Dims& d) { return d.dtype == KVM_BF16 ? KVM_MERGE_TOK_BF16 : 64; }
+static int merge_tile_tokens(const Dims& d) { return d.dtype == KVM_BF16 ? KVM_MERGE_TOK_BF16 : 32; }
 
 size_t merge_scratch_floats(const Dims& d) {
     const int TOK = merge_tile_tokens(d);
@@ -483,9 +450,9 @@ cudaError_t launch_merge(const Dims& d, const void* K, const void* V, const int3
                           : launch_t<__nv_bfloat16, 64, KVM_MERGE_TOK_BF16>(d, K, V, set_start, pivot, set_id, out_len,
                                                                          K_out, V_out, out_size, scratch, set_coef, token_d2, stats, st);
     }
-    return d.D == 128 ? launch_t<float, 128, 64>(d, K, V, set_start, pivot, set_id, out_len, K_out, V_out, out_size,
+    return d.D == 128 ? launch_t<float, 128, 32>(d, K, V, set_start, pivot, set_id, out_len, K_out, V_out, out_size,
                                                  scratch, set_coef, token_d2, stats, st)
-                      : launch_t<float, 64, 64>(d, K, V, set_start, pivot, set_id, out_len, K_out, V_out, out_size,
+                      : launch_t<float, 64, 32>(d, K, V, set_start, pivot, set_id, out_len, K_out, V_out, out_size,
                                                 scratch, set_coef, token_d2, stats, st);
 }
 
