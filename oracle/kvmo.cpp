@@ -13,7 +13,9 @@
 // Indices are 0-based.
 //
 // Parity pins (tests/test_oracle_*.py): every function below is pinned by
-// closed forms, invariants or brute force.  Parity unpinned BY THE PAPER (no
+// closed forms, invariants, library routines or brute force (kvmo_prefill_attend:
+// a library softmax row by row, the row-sum invariant, its last row against
+// kvmo_attend and its log-sum-exp against kvmo_scores).  Parity unpinned BY THE PAPER (no
 // printed example; pinned only by brute force, monotonicity and invariants):
 // the budget rule in kvmo_boundaries; the per-set bandwidth of kvmo_merge's
 // weight_rule 3 (a reading of Eq. 4, which is circular as printed).
@@ -413,6 +415,40 @@ void kvmo_attend(int32_t B, int32_t Hq, int32_t Hkv, int32_t rows, int32_t D, do
             for (int32_t j = 0; j < n; ++j)
                 for (int32_t t = 0; t < D; ++t) o[t] += (s[j] / l) * (double)Vu[(size_t)j * D + t];
         }
+}
+
+// Eq. 1 for every position of the prompt at once (the prefill): for query head h (KV head h / G) and
+// position i, O_i = sum_{j <= i} softmax_j(scale * <q_i, k_j>) v_j over the causal prefix, and the row's
+// log-sum-exp lse_i = ln sum_{j <= i} exp(scale * <q_i, k_j>) (the quantity kvmo_scores also returns).
+// Q [B,Hq,S,D], K/V [B,Hkv,S,D]; out [B,Hq,S,D]; lse (nullable) [B,Hq,S].
+void kvmo_prefill_attend(int32_t B, int32_t Hq, int32_t Hkv, int32_t S, int32_t D, double scale, const float* Q,
+                         const float* K, const float* V, double* out, double* lse) {
+    const int32_t G = Hq / Hkv;
+    for (int64_t qh = 0; qh < (int64_t)B * Hq; ++qh) {
+        const int64_t b = qh / Hq, h = qh % Hq;
+        const int64_t u = b * Hkv + h / G;
+        const float* Qh = Q + (size_t)qh * S * D;
+        const float* Ku = K + (size_t)u * S * D;
+        const float* Vu = V + (size_t)u * S * D;
+#pragma omp parallel for schedule(static, 8)
+        for (int32_t i = 0; i < S; ++i) {
+            std::vector<double> s(i + 1);
+            double m = -INFINITY;
+            for (int32_t j = 0; j <= i; ++j) {
+                double dot = 0.0;
+                for (int32_t t = 0; t < D; ++t) dot += (double)Qh[(size_t)i * D + t] * (double)Ku[(size_t)j * D + t];
+                s[j] = scale * dot;
+                m = std::max(m, s[j]);
+            }
+            double l = 0.0;
+            for (int32_t j = 0; j <= i; ++j) { s[j] = std::exp(s[j] - m); l += s[j]; }
+            double* o = out + ((size_t)qh * S + i) * D;
+            for (int32_t t = 0; t < D; ++t) o[t] = 0.0;
+            for (int32_t j = 0; j <= i; ++j)
+                for (int32_t t = 0; t < D; ++t) o[t] += (s[j] / l) * (double)Vu[(size_t)j * D + t];
+            if (lse) lse[(size_t)qh * S + i] = m + std::log(l);
+        }
+    }
 }
 
 // Definition 2.1's criterion |O_t - O_t*|, read as the Euclidean norm per

@@ -218,6 +218,21 @@ def attend(q, K, V, length=None, scale: Optional[float] = None) -> np.ndarray:
     return out
 
 
+def prefill_attend(Q, K, V, scale: Optional[float] = None):
+    """Causal attention over the whole prompt (Eq. 1 for every position): Q [B,Hq,S,D], K/V [B,Hkv,S,D] ->
+    O [B,Hq,S,D] fp64 and the rows' natural-log log-sum-exp [B,Hq,S]."""
+    Q, K, V = _f32(Q), _f32(K), _f32(V)
+    B, Hq, S, D = Q.shape
+    Hkv = K.shape[1]
+    if scale is None:
+        scale = 1.0 / math.sqrt(D)
+    out = np.empty((B, Hq, S, D), dtype=np.float64)
+    lse = np.empty((B, Hq, S), dtype=np.float64)
+    lib().kvmo_prefill_attend(ctypes.c_int32(B), ctypes.c_int32(Hq), ctypes.c_int32(Hkv), ctypes.c_int32(S),
+                              ctypes.c_int32(D), ctypes.c_double(scale), _p(Q), _p(K), _p(V), _p(out), _p(lse))
+    return out, lse
+
+
 def perturbation(O: np.ndarray, O_star: np.ndarray):
     """Definition 2.1's |O_t - O_t*| per head (Euclidean norm) and |O_t|."""
     O = np.ascontiguousarray(O, dtype=np.float64)

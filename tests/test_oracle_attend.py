@@ -81,3 +81,52 @@ def test_no_merging_means_no_perturbation_and_merging_perturbs():
     pv = st[..., :-1].copy()
     Ko, Vo = kvmo.merge(K2, V2, st, pv, np.full((1, 4), 32, np.int32), sigma=5.0, scale_v=False)
     np.testing.assert_allclose(kvmo.attend(qt, Ko, Vo), kvmo.attend(qt, K2, V2), rtol=1e-12, atol=1e-14)
+
+
+# ---------------------------------------------------------------- causal attention over the whole prompt (Eq. 1)
+def test_prefill_attend_matches_library_softmax_row_by_row_with_gqa_and_scale():
+    from scipy.special import logsumexp
+    B, Hq, Hkv, S, D = 2, 4, 2, 13, 8
+    Q, K, V = _rand((B, Hq, S, D), 20), _rand((B, Hkv, S, D), 21), _rand((B, Hkv, S, D), 22)
+    for scale in (None, 0.61):
+        O, lse = kvmo.prefill_attend(Q, K, V, scale)
+        sc = scale if scale is not None else 1 / math.sqrt(D)
+        for b in range(B):
+            for h in range(Hq):
+                g = h // 2
+                for i in range(S):
+                    logits = sc * (K[b, g, :i + 1].astype(np.float64) @ Q[b, h, i].astype(np.float64))
+                    np.testing.assert_allclose(O[b, h, i], softmax(logits) @ V[b, g, :i + 1].astype(np.float64),
+                                               rtol=1e-12, atol=1e-14)
+                    np.testing.assert_allclose(lse[b, h, i], logsumexp(logits), rtol=1e-13)
+
+
+def test_prefill_attend_invariants_and_its_links_to_the_other_steps():
+    B, Hq, Hkv, S, D = 1, 4, 2, 21, 8
+    Q, K, V = _rand((B, Hq, S, D), 23), _rand((B, Hkv, S, D), 24), _rand((B, Hkv, S, D), 25)
+    O, lse = kvmo.prefill_attend(Q, K, V)
+    # the first position sees only itself: its output is the first value row, its log-sum-exp its own logit
+    for h in range(Hq):
+        np.testing.assert_array_equal(O[0, h, 0], V[0, h // 2, 0].astype(np.float64))
+        np.testing.assert_allclose(lse[0, h, 0], (Q[0, h, 0].astype(np.float64) @ K[0, h // 2, 0]) / math.sqrt(D),
+                                   rtol=1e-14)
+    # rows of the attention map sum to one: constant values come back unchanged; outputs lie in the values' hull
+    ones = np.ones_like(V)
+    np.testing.assert_allclose(kvmo.prefill_attend(Q, K, ones)[0], 1.0, rtol=1e-13)
+    Vd = V.astype(np.float64)
+    for h in range(Hq):
+        for i in range(S):
+            assert (O[0, h, i] <= Vd[0, h // 2, :i + 1].max(0) + 1e-12).all()
+            assert (O[0, h, i] >= Vd[0, h // 2, :i + 1].min(0) - 1e-12).all()
+    # the last position is the decode step over the whole cache, and the log-sum-exp is the one the score step uses
+    np.testing.assert_allclose(O[:, :, -1], kvmo.attend(Q[:, :, -1], K, V), rtol=1e-12, atol=1e-14)
+    _, lse_scores = kvmo.scores(Q, K, want_lse=True)
+    np.testing.assert_allclose(lse, lse_scores, rtol=1e-13)
+    # a future token never matters: changing the last key and value leaves every earlier row as it was
+    K2, V2 = K.copy(), V.copy()
+    K2[:, :, -1] += 3.0
+    V2[:, :, -1] -= 2.0
+    O2, lse2 = kvmo.prefill_attend(Q, K2, V2)
+    np.testing.assert_array_equal(O2[:, :, :-1], O[:, :, :-1])
+    np.testing.assert_array_equal(lse2[:, :, :-1], lse[:, :, :-1])
+    assert not np.allclose(O2[:, :, -1], O[:, :, -1])
