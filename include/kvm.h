@@ -247,6 +247,25 @@ int kvm_layer_ratio(const kvm_params* p, const void* K, float* ratio, float* sim
                     void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * Causal attention over the whole prompt (Eq. 1 for every position: O_i = softmax_{j<=i}(q_i K^T * scale) V), the
+ * attention a prefill runs in any case, together with each row's natural-log log-sum-exp.  The compression is
+ * applied at the end of the prefill (Section 4, Figure 4): a caller that computes its prefill attention here hands
+ * `lse` to kvm_compress_with_lse (or kvm_score's lse_in) and the score step then needs no row pass of its own.
+ * Query head h of batch entry b reads KV head h / G.
+ *   Q    [batch, n_q_heads, S, D], K, V [batch, n_kv_heads, S, D]: device, bf16 (KVM_E_UNSUPPORTED otherwise),
+ *        16-byte aligned, not written
+ *   O    [batch, n_q_heads, S, D] bf16 (device), written: fp32 accumulation, one rounding at the store; the
+ *        probabilities enter the second product rounded to bf16, as in the tensor-core attention kernels in use
+ *   lse  [batch, n_q_heads, S] fp32 (device), written: ln sum_{j<=i} exp(scale * q_i.k_j)
+ *   stats NULL or a device kvm_stats: status = KVM_E_DEVICE_TIMEOUT if a bounded wait inside the kernel gave up
+ *        (the rows in hand at that moment are then NaN, rows of later work items are not written)
+ * Tensor cores (tcgen05); no workspace.  Only the shape, dtype and softmax_scale of p are used.  Enqueues on the
+ * stream and returns; errors found on the host are returned before anything is enqueued.
+ */
+int kvm_prefill_attend(const kvm_params* p, const void* Q, const void* K, const void* V, void* O, float* lse,
+                       kvm_stats* stats, void* cuda_stream);
+
+/*
  * One decode step of attention (Eq. 1: O_t = softmax(q_t K^T * scale) V) over a cache whose units may hold
  * different numbers of rows, e.g. the output of kvm_compress.  Query head h of batch entry b reads KV head h / G.
  *   q    [batch, n_q_heads, D] in p->dtype

@@ -26,7 +26,7 @@ EXPORTS = (
     "kvm_sizes", "kvm_workspace_bytes", "kvm_score", "kvm_row_lse", "kvm_segment", "kvm_merge_compact", "kvm_compress",
     "kvm_compress_with_lse",
     "kvm_host_staging_bytes", "kvm_compress_host", "kvm_score_static", "kvm_layer_ratio", "kvm_attend",
-    "kvm_output_perturbation", "kvm_status_string",
+    "kvm_output_perturbation", "kvm_prefill_attend", "kvm_status_string",
     "kvm_version",
 )
 KVM_STATIC_SCORE_ROWS = 1 << 20
@@ -174,6 +174,12 @@ def kvm_layer_ratio(p: KvmParams, K, ratio, sim_out, ws, stream=None) -> None:
 def kvm_attend(p: KvmParams, q, K, V, rows: int, length, out, ws, stream=None) -> None:
     _check(lib().kvm_attend(ctypes.byref(p), _ptr(q), _ptr(K), _ptr(V), ctypes.c_int32(rows), _ptr(length), _ptr(out),
                             _ptr(ws), ctypes.c_size_t(ws.numel() * ws.element_size()), _stream(stream)), "kvm_attend")
+
+
+def kvm_prefill_attend(p: KvmParams, Q, K, V, O, lse, stats=None, stream=None) -> None:
+    """Causal attention over the whole prompt: O [B,Hq,S,D] bf16 and the rows' natural-log log-sum-exp [B,Hq,S]."""
+    _check(lib().kvm_prefill_attend(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(lse), _ptr(stats),
+                                    _stream(stream)), "kvm_prefill_attend")
 
 
 def kvm_output_perturbation(p: KvmParams, q, K, V, K_c, V_c, len_c, out_full, out_comp, err, ref, ws,

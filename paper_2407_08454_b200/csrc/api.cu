@@ -235,6 +235,18 @@ int kvm_layer_ratio(const kvm_params* p, const void* K, float* ratio, float* sim
     return launch_set_ratio(d, sim, ratio, st) == cudaSuccess ? KVM_OK : KVM_E_CUDA;
 }
 
+int kvm_prefill_attend(const kvm_params* p, const void* Q, const void* K, const void* V, void* O, float* lse,
+                       kvm_stats* stats, void* cuda_stream) {
+    Dims d;
+    int rc = derive(p, d);
+    if (rc != KVM_OK) return rc;
+    if (d.dtype != KVM_BF16) return KVM_E_UNSUPPORTED;
+    if (!Q || !K || !V || !O || !lse) return KVM_E_NULL;
+    if (misaligned(Q) || misaligned(K) || misaligned(V) || misaligned(O)) return KVM_E_ALIGN;
+    return launch_prefill_attend(d, Q, K, V, O, lse, stats, (cudaStream_t)cuda_stream) == cudaSuccess ? KVM_OK
+                                                                                                     : KVM_E_CUDA;
+}
+
 int kvm_attend(const kvm_params* p, const void* q, const void* K, const void* V, int32_t rows, const int32_t* len,
                float* out, void* ws, size_t ws_bytes, void* cuda_stream) {
     Dims d;

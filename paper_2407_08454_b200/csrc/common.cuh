@@ -85,6 +85,8 @@ cudaError_t launch_score_tc(const Dims& d, const void* Q, const void* K, const f
                             float* scores, kvm_stats* stats, cudaStream_t st, float* sim_out = nullptr,
                             float* lse_out = nullptr);
 size_t score_tc_scratch_bytes_per_row();
+cudaError_t launch_prefill_attend(const Dims& d, const void* Q, const void* K, const void* V, void* O, float* lse,
+                                  kvm_stats* stats, cudaStream_t st);
 cudaError_t launch_similarity(const Dims& d, const void* K, float* sim, cudaStream_t st);
 cudaError_t launch_segment(const Dims& d, const float* scores, const float* sim, int32_t* set_id,
                            int32_t* set_start, int32_t* pivot, int32_t* out_len, kvm_stats* stats, cudaStream_t st);

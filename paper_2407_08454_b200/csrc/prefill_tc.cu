@@ -1,0 +1,366 @@
+// Causal attention over the whole prompt on the 5th-generation tensor cores (bf16 inputs):
+//   O_i = sum_{j<=i} softmax_j(c q_i.k_j) v_j,   lse_i = ln sum_{j<=i} exp(c q_i.k_j)          Eq. 1
+// This is the attention a prefill runs anyway; its row log-sum-exp is exactly what the score step's row pass
+// computes, so a caller that runs this kernel hands `lse` to kvm_compress_with_lse and pays for no row pass.
+//
+// A work item is one 128-row query tile of one query head with the key/value tiles 0..it it attends to.  Per
+// key tile ("step") two tcgen05.mma chains run: S = Q K^T into one of two 128-column TMEM accumulators, and
+// O += P V into a third, with P = exp(S - reference) written to shared memory as bf16 by the softmax warps in
+// the layout the tensor core reads (128-byte rows, 128-byte swizzle) and V read with its head dimension
+// contiguous (the layout it has in memory).  A softmax thread owns one query row = one TMEM lane: it keeps the
+// row's reference maximum and sum in registers, holds the 128 logits of a step in registers (the accumulator is
+// handed back at once), and multiplies the row of O by exp(old - new reference) only when the maximum has
+// grown by more than 8 (log2 units) since the reference was set, so that most steps touch O not at all.
+//
+// One CTA per SM, persistent:  warps 0-3 softmax,  warp 4 producer (TMA, 128-byte swizzle; K and V tiles in
+// rings of two),  warp 5 one thread issues the MMAs and owns tensor memory.  Items are dealt longest first,
+// boustrophedon.  Every wait on an mbarrier is bounded; a wait that runs out raises a flag, every role leaves
+// its loops, the rows in hand are written as NaN, kvm_stats.status is set when given, tensor memory is freed.
+#include <mutex>
+
+#include "tc_common.cuh"
+
+namespace kvm {
+namespace {
+
+using namespace tc;
+
+constexpr int TILE = 128;
+constexpr int KCHUNK = 64;
+constexpr int NKV = 2;                  // ring depth of the K tiles and of the V tiles
+constexpr int NSOFT = 4;                // softmax warps: one per TMEM lane quarter
+constexpr int NTHREADS = (NSOFT + 2) * 32;
+constexpr uint32_t CHUNK_BYTES = TILE * 128;            // [128 rows x 64 bf16]
+constexpr float LOG2E = 1.4426950408889634f, LN2 = 0.6931471805599453f;
+constexpr float RESCALE_STEP = 8.f;     // the reference maximum follows the running maximum in steps of at least this
+constexpr uint32_t S_COLS = TILE, O_COL0 = 2 * S_COLS;  // TMEM columns: S0 | S1 | O
+
+struct __align__(8) Bars {
+    uint64_t q_full, q_empty;
+    uint64_t k_full[NKV], k_empty[NKV], v_full[NKV], v_empty[NKV];
+    uint64_t s_full[2], s_empty[2];
+    uint64_t p_full, pv_done, o_empty;
+};
+struct alignas(16) Shared {
+    Bars bar;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+struct Sched {
+    int P, c, NH, T;
+    __device__ __forceinline__ bool item(int n, int& head, int& tile) const {
+        const long long k = (long long)n * P + ((n & 1) ? (P - 1 - c) : c);
+        if (k >= (long long)NH * T) return false;
+        head = (int)(k % NH);
+        tile = T - 1 - (int)(k / NH);
+        return true;
+    }
+};
+
+template <int KCH>
+__global__ void __launch_bounds__(NTHREADS, 1)
+prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                      const __grid_constant__ CUtensorMap map_v, __nv_bfloat16* __restrict__ O,
+                      float* __restrict__ lse, kvm_stats* stats, int B, int Hq, int Hkv, int S, float scale2) {
+    constexpr int D = KCH * KCHUNK;
+    constexpr uint32_t TILE_BYTES = KCH * CHUNK_BYTES;     // a Q, K or V tile
+    constexpr uint32_t P_BYTES = 2 * CHUNK_BYTES;          // P: [2 key chunks][128 rows][128 B]
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* aligned = smem_raw + (base - smem_u32(smem_raw));
+    uint8_t* sQ = aligned;
+    uint8_t* sK = sQ + TILE_BYTES;
+    uint8_t* sV = sK + NKV * TILE_BYTES;
+    uint8_t* sP = sV + NKV * TILE_BYTES;
+    Shared& sh = *reinterpret_cast<Shared*>(sP + P_BYTES);
+    volatile int* abort_flag = &sh.abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int G = Hq / Hkv;
+    const int T = (S + TILE - 1) / TILE;
+    const Sched sc{(int)gridDim.x, (int)blockIdx.x, B * Hq, T};
+
+    if (threadIdx.x == 0) {
+        mbar_init(&sh.bar.q_full, 1); mbar_init(&sh.bar.q_empty, 1);
+        for (int i = 0; i < NKV; ++i) {
+            mbar_init(&sh.bar.k_full[i], 1); mbar_init(&sh.bar.k_empty[i], 1);
+            mbar_init(&sh.bar.v_full[i], 1); mbar_init(&sh.bar.v_empty[i], 1);
+        }
+        for (int i = 0; i < 2; ++i) { mbar_init(&sh.bar.s_full[i], 1); mbar_init(&sh.bar.s_empty[i], NSOFT); }
+        mbar_init(&sh.bar.p_full, NSOFT); mbar_init(&sh.bar.pv_done, 1); mbar_init(&sh.bar.o_empty, NSOFT);
+        sh.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == NSOFT + 1) tmem_alloc(&sh.tmem_base, 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = sh.tmem_base;
+
+    if (warp == NSOFT) {
+        // ============================== producer ==============================
+        if (lane == 0) {
+            uint32_t kv = 0;                                  // K/V tiles loaded so far
+            bool ok = true;
+            int head, tile;
+            for (int n = 0; ok && sc.item(n, head, tile); ++n) {
+                ok = mbar_wait(&sh.bar.q_empty, (n & 1) ^ 1, abort_flag);
+                if (!ok) break;
+                mbar_expect_tx(&sh.bar.q_full, TILE_BYTES);
+#pragma unroll
+                for (int kc = 0; kc < KCH; ++kc)
+                    tma_load_3d(sQ + kc * CHUNK_BYTES, &map_q, &sh.bar.q_full, kc * KCHUNK, tile * TILE, head);
+                const int kvhead = (head / Hq) * Hkv + (head % Hq) / G;
+                for (int j = 0; j <= tile; ++j, ++kv) {
+                    const int s = kv % NKV;
+                    const uint32_t par = ((kv / NKV) & 1) ^ 1;
+                    ok = mbar_wait(&sh.bar.k_empty[s], par, abort_flag);
+                    if (!ok) break;
+                    mbar_expect_tx(&sh.bar.k_full[s], TILE_BYTES);
+#pragma unroll
+                    for (int kc = 0; kc < KCH; ++kc)
+                        tma_load_3d(sK + s * TILE_BYTES + kc * CHUNK_BYTES, &map_k, &sh.bar.k_full[s], kc * KCHUNK,
+                                    j * TILE, kvhead);
+                    ok = mbar_wait(&sh.bar.v_empty[s], par, abort_flag);
+                    if (!ok) break;
+                    mbar_expect_tx(&sh.bar.v_full[s], TILE_BYTES);
+#pragma unroll
+                    for (int kc = 0; kc < KCH; ++kc)
+                        tma_load_3d(sV + s * TILE_BYTES + kc * CHUNK_BYTES, &map_v, &sh.bar.v_full[s], kc * KCHUNK,
+                                    j * TILE, kvhead);
+                }
+            }
+            // Copies already issued complete on their own; before shared memory is given back, let them land
+            // (bounded: each try_wait suspends for a while by itself).
+            if (*abort_flag)
+                for (uint32_t it = 0; it < (1u << 14); ++it) mbar_try(&sh.bar.q_full, 0);
+        }
+    } else if (warp == NSOFT + 1) {
+        // ============================== MMA issue ==============================
+        if (lane == 0) {
+            constexpr uint32_t IDESC_S = idesc_bf16(TILE), IDESC_O = idesc_bf16(D, true);
+            const uint64_t desc_q = smem_desc(base);
+            const uint64_t desc_k0 = smem_desc(base + TILE_BYTES);
+            const uint32_t v_addr0 = base + TILE_BYTES + NKV * TILE_BYTES;
+            const uint64_t desc_p = smem_desc(v_addr0 + NKV * TILE_BYTES);
+            uint32_t ks_cnt = 0, vs_cnt = 0, s_cnt = 0, pv_cnt = 0;   // K tiles, V tiles, S buffers, PV products so far
+            bool ok = true;
+            int head, tile;
+            auto issue_s = [&]() {                           // S[s_cnt % 2] = Q K^T with the next K tile
+                const int s = ks_cnt % NKV, sb = s_cnt & 1;
+                ok = mbar_wait(&sh.bar.k_full[s], (ks_cnt / NKV) & 1, abort_flag) &&
+                     mbar_wait(&sh.bar.s_empty[sb], ((s_cnt >> 1) & 1) ^ 1, abort_flag);
+                if (!ok) return;
+                tc_fence_after();
+                const uint64_t dk = desc_k0 + (uint64_t)s * (TILE_BYTES >> 4);
+#pragma unroll
+                for (int kc = 0; kc < KCH; ++kc)
+#pragma unroll
+                    for (int ks = 0; ks < KCHUNK / 16; ++ks)
+                        umma_bf16(tmem_base + sb * S_COLS, desc_q + ((kc * CHUNK_BYTES + ks * 32) >> 4),
+                                  dk + ((kc * CHUNK_BYTES + ks * 32) >> 4), IDESC_S, (kc | ks) ? 1u : 0u);
+                umma_commit(&sh.bar.k_empty[s]);
+                umma_commit(&sh.bar.s_full[sb]);
+                ++ks_cnt; ++s_cnt;
+            };
+            for (int n = 0; ok && sc.item(n, head, tile); ++n) {
+                ok = mbar_wait(&sh.bar.q_full, n & 1, abort_flag);
+                if (!ok) break;
+                issue_s();
+                for (int j = 0; ok && j <= tile; ++j) {
+                    if (j < tile) { issue_s(); if (!ok) break; }     // the next step's logits while this step's softmax runs
+                    if (j == 0) ok = mbar_wait(&sh.bar.o_empty, (n & 1) ^ 1, abort_flag);   // the last item's O has been read
+                    const int s = vs_cnt % NKV;
+                    ok = ok && mbar_wait(&sh.bar.p_full, pv_cnt & 1, abort_flag) &&
+                         mbar_wait(&sh.bar.v_full[s], (vs_cnt / NKV) & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t va = v_addr0 + s * TILE_BYTES;
+#pragma unroll
+                    for (int kk = 0; kk < TILE / 16; ++kk)          // 16 keys per MMA
+                        umma_bf16(tmem_base + O_COL0, desc_p + (((kk / 4) * CHUNK_BYTES + (kk % 4) * 32) >> 4),
+                                  smem_desc_mn(va + kk * 16 * 128, CHUNK_BYTES), IDESC_O, (j | kk) ? 1u : 0u);
+                    umma_commit(&sh.bar.v_empty[s]);
+                    umma_commit(&sh.bar.pv_done);            // P may be overwritten, O may be read or rescaled
+                    ++vs_cnt; ++pv_cnt;
+                }
+                if (ok) umma_commit(&sh.bar.q_empty);
+            }
+        }
+    } else {
+        // ============================== softmax ==============================
+        const int row = warp * 32 + lane;                    // query row of the tile = TMEM lane
+        const uint32_t t_lane = tmem_base + ((uint32_t)(warp * 32) << 16);
+        uint32_t s_cnt = 0, pv_cnt = 0;
+        bool ok = true;
+        int head, tile;
+        for (int n = 0; ok && sc.item(n, head, tile); ++n) {
+            float m = -INFINITY, l = 0.f;                    // reference maximum (log2 units) and sum relative to it
+            for (int j = 0; j <= tile; ++j) {
+                const int sb = s_cnt & 1;
+                ok = mbar_wait(&sh.bar.s_full[sb], (s_cnt >> 1) & 1, abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                uint32_t vr[TILE];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) tmem_ld32_issue(t_lane + sb * S_COLS + q * 32, vr + q * 32);
+                tmem_ld_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh.bar.s_empty[sb]);   // the accumulator goes back at once
+                ++s_cnt;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) tmem_ld_fence(vr + q * 32);
+                float v[TILE];
+#pragma unroll
+                for (int c = 0; c < TILE; ++c) v[c] = __uint_as_float(vr[c]);
+                if (j == tile) {                             // diagonal tile: keys after the query do not exist for it
+#pragma unroll
+                    for (int c = 0; c < TILE; ++c)
+                        if (c > row) v[c] = -INFINITY;
+                }
+                float mx = v[0];
+#pragma unroll
+                for (int c = 1; c + 1 < TILE; c += 2) mx = fmax3(mx, v[c], v[c + 1]);
+                mx = fmaxf(mx, v[TILE - 1]) * scale2;
+                // the reference moves only when the maximum has outgrown it by RESCALE_STEP: exp2(x - m) stays
+                // below 2^RESCALE_STEP, and O is rescaled rarely
+                float alpha = 1.f;
+                const bool grow = mx > m + RESCALE_STEP;
+                if (j == 0) m = mx;
+                else if (grow) { alpha = ex2(m - mx); m = mx; }
+                const bool rescale = j > 0 && __any_sync(0xffffffffu, grow);
+                // p = 2^(x - m), summed in fp32, rounded to bf16 for the tensor core
+                const uint64_t sc2 = pack2(scale2, scale2), nm2 = pack2(-m, -m);
+                float sum[4] = {0.f, 0.f, 0.f, 0.f};
+                uint32_t pk[TILE / 2];
+#pragma unroll
+                for (int c = 0; c < TILE; c += 2) {
+                    float x0, x1;
+                    unpack2(ffma2(pack2(v[c], v[c + 1]), sc2, nm2), x0, x1);
+                    const float e0 = ex2(x0), e1 = ex2(x1);
+                    sum[(c >> 1) & 3] += e0 + e1;
+                    pk[c >> 1] = Vec<__nv_bfloat16>::pack2(e0, e1);
+                }
+                l = l * alpha + ((sum[0] + sum[1]) + (sum[2] + sum[3]));
+                // the previous step's P V has to be done before P is overwritten or O rescaled
+                ok = mbar_wait(&sh.bar.pv_done, (pv_cnt & 1) ^ 1, abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                if (rescale) {
+                    tc_fence_after();
+#pragma unroll
+                    for (int q = 0; q < D / 32; ++q) {
+                        uint32_t orr[32];
+                        tmem_ld32_issue(t_lane + O_COL0 + q * 32, orr);
+                        tmem_ld_wait();
+                        tmem_ld_fence(orr);
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
+                        tmem_st32(t_lane + O_COL0 + q * 32, orr);
+                    }
+                    tmem_st_wait();
+                }
+                // P row: 16-byte piece c of key chunk kc sits at piece c ^ (row & 7) of the row's 128 bytes
+                uint8_t* prow = sP + row * 128;
+#pragma unroll
+                for (int c = 0; c < 16; ++c) {
+                    const int kc = c >> 3, piece = c & 7;
+                    *reinterpret_cast<uint4*>(prow + kc * CHUNK_BYTES + ((piece ^ (row & 7)) << 4)) =
+                        make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+                }
+                fence_proxy_async();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh.bar.p_full);
+                ++pv_cnt;
+            }
+            // ---- item end: O / l and the row's log-sum-exp
+            const int gi = tile * TILE + row;
+            if (ok) {
+                ok = mbar_wait(&sh.bar.pv_done, (pv_cnt & 1) ^ 1, abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+            }
+            __nv_bfloat16* orow = O + ((size_t)head * S + gi) * D;
+            if (ok) {
+                tc_fence_after();
+                const float inv = 1.f / l;
+#pragma unroll
+                for (int q = 0; q < D / 32; ++q) {
+                    uint32_t orr[32];
+                    tmem_ld32_issue(t_lane + O_COL0 + q * 32, orr);
+                    tmem_ld_wait();
+                    tmem_ld_fence(orr);
+                    if (gi < S) {
+#pragma unroll
+                        for (int c = 0; c < 32; c += 8) {
+                            float f[8];
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(orr[c + e]) * inv;
+                            *reinterpret_cast<uint4*>(orow + q * 32 + c) = Vec<__nv_bfloat16>::pack(f);
+                        }
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh.bar.o_empty);
+                if (gi < S) lse[(size_t)head * S + gi] = (m + log2f(l)) * LN2;
+            } else if (gi < S) {
+                // a wait gave up: what this row would have received is marked, not made up
+                for (int c = 0; c < D; c += 8)
+                    *reinterpret_cast<uint4*>(orow + c) = make_uint4(0x7FC07FC0u, 0x7FC07FC0u, 0x7FC07FC0u, 0x7FC07FC0u);
+                lse[(size_t)head * S + gi] = NAN;
+            }
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0 && sh.abort_flag && stats) stats->status = KVM_E_DEVICE_TIMEOUT;
+    if (warp == NSOFT + 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+template <int KCH>
+cudaError_t launch_t(const Dims& d, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
+                     __nv_bfloat16* O, float* lse, kvm_stats* stats, cudaStream_t st) {
+    const size_t smem = 1024 + (size_t)(1 + 2 * NKV) * KCH * CHUNK_BYTES + 2 * CHUNK_BYTES + sizeof(Shared);
+    static std::mutex mu;
+    static int sms_of[KVM_MAX_DEVICES] = {};
+    cudaError_t e;
+    int dev = 0, sms = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    if (dev < 0 || dev >= KVM_MAX_DEVICES) return cudaErrorInvalidDevice;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        if (!sms_of[dev]) {
+            e = cudaFuncSetAttribute(prefill_attend_kernel<KCH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+            if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+            sms_of[dev] = sms;
+        }
+        sms = sms_of[dev];
+    }
+    const int T = (d.S + TILE - 1) / TILE;
+    const long long items = (long long)d.B * d.Hq * T;
+    const int grid = (int)(items < sms ? items : sms);
+    prefill_attend_kernel<KCH><<<grid, NTHREADS, smem, st>>>(mq, mk, mv, O, lse, stats, d.B, d.Hq, d.Hkv, d.S,
+                                                            d.scale * LOG2E);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_prefill_attend(const Dims& d, const void* Q, const void* K, const void* V, void* O, float* lse,
+                                  kvm_stats* stats, cudaStream_t st) {
+    CUtensorMap mq, mk, mv;
+    if (!make_map(&mq, Q, d.B * d.Hq, d.S, d.D) || !make_map(&mk, K, d.B * d.Hkv, d.S, d.D) ||
+        !make_map(&mv, V, d.B * d.Hkv, d.S, d.D))
+        return cudaErrorNotSupported;
+    __nv_bfloat16* Ob = reinterpret_cast<__nv_bfloat16*>(O);
+    return d.D == 128 ? launch_t<2>(d, mq, mk, mv, Ob, lse, stats, st) : launch_t<1>(d, mq, mk, mv, Ob, lse, stats, st);
+}
+
+}  // namespace kvm
