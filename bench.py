@@ -433,6 +433,22 @@ def main():
         lambda i: kvm.kvm_compress_with_lse(p, bufs[i % N_BUFFERS]["Q"], bufs[i % N_BUFFERS]["K"],
                                             bufs[i % N_BUFFERS]["V"], lses[i % N_BUFFERS], comp.K_out, comp.V_out,
                                             comp.out_len, comp.out_pos, None, None, ws, stream), min(reps, 50))
+    # the prefill attention that hands over that log-sum-exp (Eq. 1 over the whole prompt), alone and followed
+    # by the compression that uses its lse; and today's alternative, the same attention followed by kvm_compress
+    o_att = torch.empty_like(b0["Q"])
+    lse_att = torch.empty(cfg.batch, cfg.n_q_heads, cfg.seq, device=dev)
+    def attend_then(i, with_lse):
+        b = bufs[i % N_BUFFERS]
+        kvm.kvm_prefill_attend(p, b["Q"], b["K"], b["V"], o_att, lse_att, None, stream)
+        if with_lse is None:
+            return
+        kvm.kvm_compress_with_lse(p, b["Q"], b["K"], b["V"], lse_att if with_lse else None, comp.K_out, comp.V_out,
+                                  comp.out_len, comp.out_pos, None, None, ws, stream)
+    t_pre = timed(lambda i: attend_then(i, None), min(reps, 50))
+    extras["prefill_attend_ms"] = t_pre
+    extras["prefill_attend_tflops"] = 2 * work["flops_per_score_pass"] / (t_pre * 1e-3) / 1e12
+    extras["prefill_attend_then_compress_with_lse_ms"] = timed(lambda i: attend_then(i, True), min(reps, 50))
+    extras["prefill_attend_then_compress_ms"] = timed(lambda i: attend_then(i, False), min(reps, 50))
     ratio = torch.empty(U, device=dev)
     extras["layer_ratio_ms"] = timed(lambda i: kvm.kvm_layer_ratio(p, bufs[i % N_BUFFERS]["K"], ratio, None, ws,
                                                                    stream), min(reps, 50))
