@@ -220,6 +220,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-workloads", action="store_true", help="skip the C2-C4 section of extras")
+    ap.add_argument("--min-ms", type=float, default=MIN_TIMED_MS,
+                    help="GPU time to accumulate over repeated timed blocks (profiler captures use a small value)")
     args = ap.parse_args()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         raise SystemExit(spawn_ranks(args.gpus))
@@ -273,7 +275,7 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    def timed_blocks(fn, steps, min_ms=MIN_TIMED_MS, max_blocks=400):
+    def timed_blocks(fn, steps, min_ms=args.min_ms, max_blocks=400):
         """Blocks of `steps` calls between two events each, repeated until min_ms of GPU time; every rank runs the
         same number of blocks (the count is fixed from the first block's slowest-rank time)."""
         def one_block():
@@ -302,7 +304,7 @@ def main():
     st = kvm.read_stats(stats)
     assert st.status == 0, "device reported an error status"
     # the same step on one input set that stays in L2 between calls (the working set of a layer is of L2's size)
-    warm_ms = timed_blocks(lambda i: step(i, rotate=False), args.steps, min_ms=100.0)
+    warm_ms = timed_blocks(lambda i: step(i, rotate=False), args.steps, min_ms=min(100.0, args.min_ms))
     l2_warm = stats_of([b / args.steps for b in warm_ms])
 
     # ---- per-kernel timing (same launches, event pairs around each public step)
@@ -485,7 +487,7 @@ def main():
 
     for i in range(3):
         host_step(i)
-    e2e_blocks = timed_blocks(host_step, e2e_steps, min_ms=300.0, max_blocks=20)
+    e2e_blocks = timed_blocks(host_step, e2e_steps, min_ms=min(300.0, args.min_ms), max_blocks=20)
     ms_e2e = sum(e2e_blocks) / len(e2e_blocks)
     assert int(hlen.sum()) > 0, "the host path returned no rows"
     esz = 2 if cfg.dtype == "bf16" else 4
