@@ -4,18 +4,22 @@
 // computes, so a caller that runs this kernel hands `lse` to kvm_compress_with_lse and pays for no row pass.
 //
 // A work item is one 128-row query tile of one query head with the key/value tiles 0..it it attends to.  Per
-// key tile ("step") two tcgen05.mma chains run: S = Q K^T into one of two 128-column TMEM accumulators, and
-// O += P V into a third, with P = exp(S - reference) written to shared memory as bf16 by the softmax warps in
-// the layout the tensor core reads (128-byte rows, 128-byte swizzle) and V read with its head dimension
-// contiguous (the layout it has in memory).  A softmax thread owns one query row = one TMEM lane: it keeps the
-// row's reference maximum and sum in registers, holds the 128 logits of a step in registers (the accumulator is
-// handed back at once), and multiplies the row of O by exp(old - new reference) only when the maximum has
-// grown by more than 8 (log2 units) since the reference was set, so that most steps touch O not at all.
+// key tile ("step") two tcgen05.mma chains run: S = Q K^T into a 128-column TMEM accumulator, and O += P V into
+// another, with P = exp(S - reference) written to shared memory as bf16 by the softmax warps in the layout the
+// tensor core reads (128-byte rows, 128-byte swizzle) and V read with its head dimension contiguous (the layout
+// it has in memory).  Two groups of four softmax warps take alternate steps, each with its own S accumulator, P
+// tile, O accumulator, reference maximum and row sum, so that one group's exponentials run under the other
+// group's products; the two partial results of a row are joined when the item ends.  A softmax thread owns one
+// query row = one TMEM lane: it holds the 128 logits of a step in registers (the accumulator is handed back at
+// once), and multiplies its row of O by exp(old - new reference) only when the maximum has grown by more than
+// 8 (log2 units) since the reference was set, so that most steps touch O not at all.
 //
-// One CTA per SM, persistent:  warps 0-3 softmax,  warp 4 producer (TMA, 128-byte swizzle; K and V tiles in
-// rings of two),  warp 5 one thread issues the MMAs and owns tensor memory.  Items are dealt longest first,
-// boustrophedon.  Every wait on an mbarrier is bounded; a wait that runs out raises a flag, every role leaves
-// its loops, the rows in hand are written as NaN, kvm_stats.status is set when given, tensor memory is freed.
+// One CTA per SM, persistent:  warps 0-7 softmax (group = warp / 4),  warp 8 producer (TMA, 128-byte swizzle; K
+// and V tiles in rings of two),  warp 9 one thread issues the MMAs and owns tensor memory (warps 10-11 only fill the
+// third warpgroup, which gives registers up to the softmax warpgroups).  Items are dealt
+// longest first, boustrophedon.  Every wait on an mbarrier is bounded; a wait that runs out raises a flag, every
+// role leaves its loops, the rows in hand are written as NaN, kvm_stats.status is set when given, tensor memory
+// is freed.
 #include <mutex>
 
 #include "tc_common.cuh"
@@ -28,23 +32,29 @@ using namespace tc;
 constexpr int TILE = 128;
 constexpr int KCHUNK = 64;
 constexpr int NKV = 2;                  // ring depth of the K tiles and of the V tiles
-constexpr int NSOFT = 4;                // softmax warps: one per TMEM lane quarter
-constexpr int NTHREADS = (NSOFT + 2) * 32;
+constexpr int NGRP = 2;                 // softmax groups taking alternate steps
+constexpr int NSOFT = 4 * NGRP;         // softmax warps: one per TMEM lane quarter and group
+constexpr int NTHREADS = (NSOFT + 4) * 32;   // three warpgroups: two of softmax warps, one with producer, MMA issue and two idle warps
+// Registers: the launch gives every thread 168 (65536 / 384); the softmax warpgroups then take 208 each and the
+// third warpgroup keeps 56 (2 x 128 x 208 + 128 x 56 = 60416 <= 384 x 168 = 64512).
+constexpr int REGS_SOFTMAX = 208, REGS_OTHER = 56;
 constexpr uint32_t CHUNK_BYTES = TILE * 128;            // [128 rows x 64 bf16]
 constexpr float LOG2E = 1.4426950408889634f, LN2 = 0.6931471805599453f;
 constexpr float RESCALE_STEP = 8.f;     // the reference maximum follows the running maximum in steps of at least this
-constexpr uint32_t S_COLS = TILE, O_COL0 = 2 * S_COLS;  // TMEM columns: S0 | S1 | O
+constexpr uint32_t S_COLS = TILE, O_COL0 = NGRP * S_COLS;  // TMEM columns: S of group 0 | S of group 1 | O 0 | O 1
 
 struct __align__(8) Bars {
     uint64_t q_full, q_empty;
     uint64_t k_full[NKV], k_empty[NKV], v_full[NKV], v_empty[NKV];
-    uint64_t s_full[2], s_empty[2];
-    uint64_t p_full, pv_done, o_empty;
+    uint64_t s_full[NGRP], s_empty[NGRP];
+    uint64_t p_full[NGRP], pv_done[NGRP], o_empty;
+    uint64_t part_full, part_empty;     // group 1's row state at item end: written / read
 };
 struct alignas(16) Shared {
     Bars bar;
     uint32_t tmem_base;
     int abort_flag;
+    float part_m[TILE], part_l[TILE];   // group 1's row state at item end (handed over through part_full / part_empty)
 };
 
 struct Sched {
@@ -72,8 +82,8 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
     uint8_t* sQ = aligned;
     uint8_t* sK = sQ + TILE_BYTES;
     uint8_t* sV = sK + NKV * TILE_BYTES;
-    uint8_t* sP = sV + NKV * TILE_BYTES;
-    Shared& sh = *reinterpret_cast<Shared*>(sP + P_BYTES);
+    uint8_t* sP = sV + NKV * TILE_BYTES;                   // one P tile per group
+    Shared& sh = *reinterpret_cast<Shared*>(sP + NGRP * P_BYTES);
     volatile int* abort_flag = &sh.abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -87,8 +97,12 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
             mbar_init(&sh.bar.k_full[i], 1); mbar_init(&sh.bar.k_empty[i], 1);
             mbar_init(&sh.bar.v_full[i], 1); mbar_init(&sh.bar.v_empty[i], 1);
         }
-        for (int i = 0; i < 2; ++i) { mbar_init(&sh.bar.s_full[i], 1); mbar_init(&sh.bar.s_empty[i], NSOFT); }
-        mbar_init(&sh.bar.p_full, NSOFT); mbar_init(&sh.bar.pv_done, 1); mbar_init(&sh.bar.o_empty, NSOFT);
+        for (int i = 0; i < NGRP; ++i) {
+            mbar_init(&sh.bar.s_full[i], 1); mbar_init(&sh.bar.s_empty[i], 4);
+            mbar_init(&sh.bar.p_full[i], 4); mbar_init(&sh.bar.pv_done[i], 1);
+        }
+        mbar_init(&sh.bar.o_empty, 4);
+        mbar_init(&sh.bar.part_full, 4); mbar_init(&sh.bar.part_empty, 4);
         sh.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -98,7 +112,9 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
     tc_fence_after();
     const uint32_t tmem_base = sh.tmem_base;
 
-    if (warp == NSOFT) {
+    if (warp >= NSOFT) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_OTHER));
+      if (warp == NSOFT) {
         // ============================== producer ==============================
         if (lane == 0) {
             uint32_t kv = 0;                                  // K/V tiles loaded so far
@@ -136,21 +152,22 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
             if (*abort_flag)
                 for (uint32_t it = 0; it < (1u << 14); ++it) mbar_try(&sh.bar.q_full, 0);
         }
-    } else if (warp == NSOFT + 1) {
+      } else if (warp == NSOFT + 1) {
         // ============================== MMA issue ==============================
         if (lane == 0) {
             constexpr uint32_t IDESC_S = idesc_bf16(TILE), IDESC_O = idesc_bf16(D, true);
             const uint64_t desc_q = smem_desc(base);
             const uint64_t desc_k0 = smem_desc(base + TILE_BYTES);
             const uint32_t v_addr0 = base + TILE_BYTES + NKV * TILE_BYTES;
-            const uint64_t desc_p = smem_desc(v_addr0 + NKV * TILE_BYTES);
-            uint32_t ks_cnt = 0, vs_cnt = 0, s_cnt = 0, pv_cnt = 0;   // K tiles, V tiles, S buffers, PV products so far
+            const uint64_t desc_p0 = smem_desc(v_addr0 + NKV * TILE_BYTES);
+            uint32_t ks_cnt = 0, vs_cnt = 0;                 // K tiles and V tiles consumed so far
+            uint32_t s_cnt[NGRP] = {0, 0}, pv_cnt[NGRP] = {0, 0};   // per group: S tiles produced, P V products issued
             bool ok = true;
             int head, tile;
-            auto issue_s = [&]() {                           // S[s_cnt % 2] = Q K^T with the next K tile
-                const int s = ks_cnt % NKV, sb = s_cnt & 1;
+            auto issue_s = [&](int g) {                      // S of group g = Q K^T with the next K tile
+                const int s = ks_cnt % NKV;
                 ok = mbar_wait(&sh.bar.k_full[s], (ks_cnt / NKV) & 1, abort_flag) &&
-                     mbar_wait(&sh.bar.s_empty[sb], ((s_cnt >> 1) & 1) ^ 1, abort_flag);
+                     mbar_wait(&sh.bar.s_empty[g], (s_cnt[g] & 1) ^ 1, abort_flag);
                 if (!ok) return;
                 tc_fence_after();
                 const uint64_t dk = desc_k0 + (uint64_t)s * (TILE_BYTES >> 4);
@@ -158,58 +175,66 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                 for (int kc = 0; kc < KCH; ++kc)
 #pragma unroll
                     for (int ks = 0; ks < KCHUNK / 16; ++ks)
-                        umma_bf16(tmem_base + sb * S_COLS, desc_q + ((kc * CHUNK_BYTES + ks * 32) >> 4),
+                        umma_bf16(tmem_base + g * S_COLS, desc_q + ((kc * CHUNK_BYTES + ks * 32) >> 4),
                                   dk + ((kc * CHUNK_BYTES + ks * 32) >> 4), IDESC_S, (kc | ks) ? 1u : 0u);
                 umma_commit(&sh.bar.k_empty[s]);
-                umma_commit(&sh.bar.s_full[sb]);
-                ++ks_cnt; ++s_cnt;
+                umma_commit(&sh.bar.s_full[g]);
+                ++ks_cnt; ++s_cnt[g];
             };
             for (int n = 0; ok && sc.item(n, head, tile); ++n) {
                 ok = mbar_wait(&sh.bar.q_full, n & 1, abort_flag);
                 if (!ok) break;
-                issue_s();
+                issue_s(0);                                  // the logits run two steps ahead of the P V products,
+                if (ok && tile >= 1) issue_s(1);             // one step per group
                 for (int j = 0; ok && j <= tile; ++j) {
-                    if (j < tile) { issue_s(); if (!ok) break; }     // the next step's logits while this step's softmax runs
+                    const int g = j & 1;
                     if (j == 0) ok = mbar_wait(&sh.bar.o_empty, (n & 1) ^ 1, abort_flag);   // the last item's O has been read
                     const int s = vs_cnt % NKV;
-                    ok = ok && mbar_wait(&sh.bar.p_full, pv_cnt & 1, abort_flag) &&
+                    ok = ok && mbar_wait(&sh.bar.p_full[g], pv_cnt[g] & 1, abort_flag) &&
                          mbar_wait(&sh.bar.v_full[s], (vs_cnt / NKV) & 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t va = v_addr0 + s * TILE_BYTES;
+                    const uint64_t dp = desc_p0 + (uint64_t)g * (P_BYTES >> 4);
 #pragma unroll
                     for (int kk = 0; kk < TILE / 16; ++kk)          // 16 keys per MMA
-                        umma_bf16(tmem_base + O_COL0, desc_p + (((kk / 4) * CHUNK_BYTES + (kk % 4) * 32) >> 4),
-                                  smem_desc_mn(va + kk * 16 * 128, CHUNK_BYTES), IDESC_O, (j | kk) ? 1u : 0u);
+                        umma_bf16(tmem_base + O_COL0 + g * S_COLS, dp + (((kk / 4) * CHUNK_BYTES + (kk % 4) * 32) >> 4),
+                                  smem_desc_mn(va + kk * 16 * 128, CHUNK_BYTES), IDESC_O, ((j >> 1) | kk) ? 1u : 0u);
                     umma_commit(&sh.bar.v_empty[s]);
-                    umma_commit(&sh.bar.pv_done);            // P may be overwritten, O may be read or rescaled
-                    ++vs_cnt; ++pv_cnt;
+                    umma_commit(&sh.bar.pv_done[g]);         // the group's P may be overwritten, its O read or rescaled
+                    ++vs_cnt; ++pv_cnt[g];
+                    if (j + 2 <= tile) issue_s(g);           // the group has taken its logits into registers long ago
                 }
                 if (ok) umma_commit(&sh.bar.q_empty);
             }
         }
+      }
     } else {
         // ============================== softmax ==============================
-        const int row = warp * 32 + lane;                    // query row of the tile = TMEM lane
-        const uint32_t t_lane = tmem_base + ((uint32_t)(warp * 32) << 16);
-        uint32_t s_cnt = 0, pv_cnt = 0;
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS_SOFTMAX));
+        const int grp = warp >> 2, lq = warp & 3;
+        const int row = lq * 32 + lane;                      // query row of the tile = TMEM lane
+        const uint32_t t_lane = tmem_base + ((uint32_t)(lq * 32) << 16);
+        const uint32_t t_s = t_lane + grp * S_COLS, t_o = t_lane + O_COL0 + grp * S_COLS;
+        uint8_t* prow = sP + grp * P_BYTES + row * 128;
+        uint32_t s_cnt = 0, pv_cnt = 0;                      // this group's steps so far
+        uint32_t pv_other = 0;                               // the other group's (group 0 reads both results at item end)
         bool ok = true;
         int head, tile;
         for (int n = 0; ok && sc.item(n, head, tile); ++n) {
             float m = -INFINITY, l = 0.f;                    // reference maximum (log2 units) and sum relative to it
-            for (int j = 0; j <= tile; ++j) {
-                const int sb = s_cnt & 1;
-                ok = mbar_wait(&sh.bar.s_full[sb], (s_cnt >> 1) & 1, abort_flag);
+            for (int j = grp; j <= tile; j += NGRP) {
+                ok = mbar_wait(&sh.bar.s_full[grp], s_cnt & 1, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after();
                 uint32_t vr[TILE];
 #pragma unroll
-                for (int q = 0; q < 4; ++q) tmem_ld32_issue(t_lane + sb * S_COLS + q * 32, vr + q * 32);
+                for (int q = 0; q < 4; ++q) tmem_ld32_issue(t_s + q * 32, vr + q * 32);
                 tmem_ld_wait();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&sh.bar.s_empty[sb]);   // the accumulator goes back at once
+                if (lane == 0) mbar_arrive(&sh.bar.s_empty[grp]);   // the accumulator goes back at once
                 ++s_cnt;
 #pragma unroll
                 for (int q = 0; q < 4; ++q) tmem_ld_fence(vr + q * 32);
@@ -228,10 +253,11 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                 // the reference moves only when the maximum has outgrown it by RESCALE_STEP: exp2(x - m) stays
                 // below 2^RESCALE_STEP, and O is rescaled rarely
                 float alpha = 1.f;
+                const bool first = j == grp;                 // the group's first step of the item
                 const bool grow = mx > m + RESCALE_STEP;
-                if (j == 0) m = mx;
+                if (first) m = mx;
                 else if (grow) { alpha = ex2(m - mx); m = mx; }
-                const bool rescale = j > 0 && __any_sync(0xffffffffu, grow);
+                const bool rescale = !first && __any_sync(0xffffffffu, grow);
                 // p = 2^(x - m), summed in fp32, rounded to bf16 for the tensor core
                 const uint64_t sc2 = pack2(scale2, scale2), nm2 = pack2(-m, -m);
                 float sum[4] = {0.f, 0.f, 0.f, 0.f};
@@ -245,8 +271,8 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                     pk[c >> 1] = Vec<__nv_bfloat16>::pack2(e0, e1);
                 }
                 l = l * alpha + ((sum[0] + sum[1]) + (sum[2] + sum[3]));
-                // the previous step's P V has to be done before P is overwritten or O rescaled
-                ok = mbar_wait(&sh.bar.pv_done, (pv_cnt & 1) ^ 1, abort_flag);
+                // the group's previous P V has to be done before its P is overwritten or its O rescaled
+                ok = mbar_wait(&sh.bar.pv_done[grp], (pv_cnt & 1) ^ 1, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 if (rescale) {
@@ -254,17 +280,16 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
 #pragma unroll
                     for (int q = 0; q < D / 32; ++q) {
                         uint32_t orr[32];
-                        tmem_ld32_issue(t_lane + O_COL0 + q * 32, orr);
+                        tmem_ld32_issue(t_o + q * 32, orr);
                         tmem_ld_wait();
                         tmem_ld_fence(orr);
 #pragma unroll
                         for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
-                        tmem_st32(t_lane + O_COL0 + q * 32, orr);
+                        tmem_st32(t_o + q * 32, orr);
                     }
                     tmem_st_wait();
                 }
                 // P row: 16-byte piece c of key chunk kc sits at piece c ^ (row & 7) of the row's 128 bytes
-                uint8_t* prow = sP + row * 128;
 #pragma unroll
                 for (int c = 0; c < 16; ++c) {
                     const int kc = c >> 3, piece = c & 7;
@@ -274,31 +299,62 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                 fence_proxy_async();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&sh.bar.p_full);
+                if (lane == 0) mbar_arrive(&sh.bar.p_full[grp]);
                 ++pv_cnt;
             }
-            // ---- item end: O / l and the row's log-sum-exp
-            const int gi = tile * TILE + row;
+            const int n_other = (tile + 1 + grp) / 2;        // steps the other group takes in this item
+            pv_other += n_other;
+            // ---- item end: group 1 hands its row state to group 0, which joins the two partial results:
+            //      O = (O_0 2^(m_0 - M) + O_1 2^(m_1 - M)) / (l_0 2^(m_0 - M) + l_1 2^(m_1 - M)),  M = max(m_0, m_1)
+            if (grp == 1) {
+                // (every item, also one in which this group had no step: the two groups count items alike)
+                ok = ok && mbar_wait(&sh.bar.part_empty, (n & 1) ^ 1, abort_flag);   // group 0 has read the last item's
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                sh.part_m[row] = m;
+                sh.part_l[row] = l;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh.bar.part_full);
+                continue;
+            }
             if (ok) {
-                ok = mbar_wait(&sh.bar.pv_done, (pv_cnt & 1) ^ 1, abort_flag);
+                ok = mbar_wait(&sh.bar.part_full, n & 1, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
             }
+            const float m1 = ok ? sh.part_m[row] : -INFINITY, l1 = ok ? sh.part_l[row] : 0.f;
+            __syncwarp();
+            if (ok && lane == 0) mbar_arrive(&sh.bar.part_empty);
+            const int gi = tile * TILE + row;
+            if (ok) {
+                ok = mbar_wait(&sh.bar.pv_done[0], (pv_cnt & 1) ^ 1, abort_flag);
+                if (ok && n_other > 0) ok = mbar_wait(&sh.bar.pv_done[1], (pv_other & 1) ^ 1, abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+            }
+            ok = ok && (*abort_flag == 0);
             __nv_bfloat16* orow = O + ((size_t)head * S + gi) * D;
             if (ok) {
                 tc_fence_after();
-                const float inv = 1.f / l;
+                const float M = fmaxf(m, m1);
+                const float w0 = ex2(m - M), w1 = n_other > 0 ? ex2(m1 - M) : 0.f;
+                const float L = l * w0 + l1 * w1;
+                const float f0 = w0 / L, f1 = w1 / L;
 #pragma unroll
                 for (int q = 0; q < D / 32; ++q) {
-                    uint32_t orr[32];
-                    tmem_ld32_issue(t_lane + O_COL0 + q * 32, orr);
+                    uint32_t o0[32], o1[32];
+                    tmem_ld32_issue(t_lane + O_COL0 + q * 32, o0);
+                    if (n_other > 0) tmem_ld32_issue(t_lane + O_COL0 + S_COLS + q * 32, o1);
                     tmem_ld_wait();
-                    tmem_ld_fence(orr);
+                    tmem_ld_fence(o0);
+                    if (n_other > 0) tmem_ld_fence(o1);
                     if (gi < S) {
 #pragma unroll
                         for (int c = 0; c < 32; c += 8) {
                             float f[8];
 #pragma unroll
-                            for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(orr[c + e]) * inv;
+                            for (int e = 0; e < 8; ++e) {
+                                f[e] = __uint_as_float(o0[c + e]) * f0;
+                                if (n_other > 0) f[e] = fmaf(__uint_as_float(o1[c + e]), f1, f[e]);
+                            }
                             *reinterpret_cast<uint4*>(orow + q * 32 + c) = Vec<__nv_bfloat16>::pack(f);
                         }
                     }
@@ -306,7 +362,7 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh.bar.o_empty);
-                if (gi < S) lse[(size_t)head * S + gi] = (m + log2f(l)) * LN2;
+                if (gi < S) lse[(size_t)head * S + gi] = (M + log2f(L)) * LN2;
             } else if (gi < S) {
                 // a wait gave up: what this row would have received is marked, not made up
                 for (int c = 0; c < D; c += 8)
@@ -326,7 +382,7 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
 template <int KCH>
 cudaError_t launch_t(const Dims& d, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                      __nv_bfloat16* O, float* lse, kvm_stats* stats, cudaStream_t st) {
-    const size_t smem = 1024 + (size_t)(1 + 2 * NKV) * KCH * CHUNK_BYTES + 2 * CHUNK_BYTES + sizeof(Shared);
+    const size_t smem = 1024 + (size_t)(1 + 2 * NKV) * KCH * CHUNK_BYTES + NGRP * 2 * CHUNK_BYTES + sizeof(Shared);
     static std::mutex mu;
     static int sms_of[KVM_MAX_DEVICES] = {};
     cudaError_t e;
