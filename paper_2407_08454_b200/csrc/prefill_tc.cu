@@ -19,7 +19,8 @@
 // third warpgroup, which gives registers up to the softmax warpgroups).  Items are dealt
 // longest first, boustrophedon.  Every wait on an mbarrier is bounded; a wait that runs out raises a flag, every
 // role leaves its loops, the rows in hand are written as NaN, kvm_stats.status is set when given, tensor memory
-// is freed.
+// is freed.  (The test build of the library, never shipped, shortens the limit and makes the producer leave out one
+// V tile, so that this path can be exercised: KVM_TEST_WAIT_LIMIT_CLOCKS, KVM_TEST_DROP_B_STAGE.)
 #include <mutex>
 
 #include "tc_common.cuh"
@@ -138,6 +139,9 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                     for (int kc = 0; kc < KCH; ++kc)
                         tma_load_3d(sK + s * TILE_BYTES + kc * CHUNK_BYTES, &map_k, &sh.bar.k_full[s], kc * KCHUNK,
                                     j * TILE, kvhead);
+#ifdef KVM_TEST_DROP_B_STAGE
+                    if (kv == (uint32_t)(KVM_TEST_DROP_B_STAGE)) continue;   // test build only: this V tile never arrives
+#endif
                     ok = mbar_wait(&sh.bar.v_empty[s], par, abort_flag);
                     if (!ok) break;
                     mbar_expect_tx(&sh.bar.v_full[s], TILE_BYTES);

@@ -55,3 +55,34 @@ def test_a_wait_that_runs_out_is_reported_and_the_next_call_is_correct():
     ref = kvmo.scores(d["Q"].double().numpy(), d["K"].double().numpy(), f32(1.0 / np.sqrt(np.float32(cfg.head_dim))))
     g = good.cpu().numpy().astype(np.float64)
     assert np.all(np.abs(g - ref) <= SCORE_RTOL * np.abs(ref) + SCORE_ATOL)
+
+
+def test_the_prefill_attention_kernel_also_comes_back_and_reports():
+    """Same build, the attention kernel: its producer leaves out the fourth V tile of every work item that has one,
+    the MMA thread's wait for it runs out, the kernel returns, the status is set, the rows that were in hand are NaN
+    and the work items that never needed that tile are complete."""
+    from oracle import kvmo
+    lib = ctypes.CDLL(build.build_waittest())
+    cfg = si.CONFIGS["C1"].scaled(seq=1024, n_q_heads=4, n_kv_heads=4, seed=78)     # 8 query tiles per head, one per CTA
+    d = si.make_layer(cfg)
+    Q, K, V = d["Q"].cuda(), d["K"].cuda(), d["V"].cuda()
+    p = kvm.make_params(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.seq, cfg.head_dim, cfg.torch_dtype)
+    O = torch.zeros_like(Q)
+    lse = torch.zeros(1, 4, 1024, device="cuda")
+    stats = kvm.new_stats("cuda")
+    vp = ctypes.c_void_p
+    rc = lib.kvm_prefill_attend(ctypes.byref(p), vp(Q.data_ptr()), vp(K.data_ptr()), vp(V.data_ptr()), vp(O.data_ptr()),
+                                vp(lse.data_ptr()), vp(stats.data_ptr()), vp(torch.cuda.current_stream().cuda_stream))
+    assert rc == 0
+    torch.cuda.synchronize()                        # the kernel came back by itself
+    assert kvm.read_stats(stats).status == -9       # KVM_E_DEVICE_TIMEOUT
+    bad = torch.isnan(lse)
+    assert bad[:, :, 3 * 128:].all()                # query tiles 3..7 need a fourth V tile: marked, not made up
+    assert not bad[:, :, :3 * 128].any()            # tiles 0..2 never needed it
+    refO, ref_lse = kvmo.prefill_attend(d["Q"][:, :, :384], d["K"][:, :, :384], d["V"][:, :, :384])
+    assert np.abs(lse[:, :, :384].cpu().numpy() - ref_lse).max() <= 2e-4
+    # the context is intact: the shipped library computes the same layer correctly right afterwards
+    kvm.kvm_prefill_attend(p, Q, K, V, O, lse)
+    torch.cuda.synchronize()
+    refO, ref_lse = kvmo.prefill_attend(d["Q"], d["K"], d["V"])
+    assert torch.isfinite(lse).all() and np.abs(lse.cpu().numpy() - ref_lse).max() <= 2e-4
