@@ -247,6 +247,21 @@ int kvm_layer_ratio(const kvm_params* p, const void* K, float* ratio, float* sim
                     void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * A stack of layers with one similarity threshold each (Section 3.2: the layer-wise compression ratios can be set
+ * by adjusting the threshold layer by layer): n_layers calls of kvm_compress, layer l with sim_threshold =
+ * sim_thresholds[l] (p->sim_threshold for all layers when sim_thresholds is NULL), enqueued one after the other on
+ * the stream; the workspace is shared, the layers' tensors are not.
+ *   Q, K, V, K_out, V_out, out_len, out_pos: HOST arrays of n_layers device pointers, each as in kvm_compress
+ *   sim_thresholds: NULL or a HOST array of n_layers floats (read before the call returns)
+ *   stats: NULL or one device kvm_stats that accumulates over the layers
+ * Every layer's arguments are checked before anything is enqueued.
+ */
+int kvm_compress_layers(const kvm_params* p, int32_t n_layers, const float* sim_thresholds, const void* const* Q,
+                        const void* const* K, const void* const* V, void* const* K_out, void* const* V_out,
+                        int32_t* const* out_len, int32_t* const* out_pos, kvm_stats* stats, void* ws,
+                        size_t ws_bytes, void* cuda_stream);
+
+/*
  * Causal attention over the whole prompt (Eq. 1 for every position: O_i = softmax_{j<=i}(q_i K^T * scale) V), the
  * attention a prefill runs in any case, together with each row's natural-log log-sum-exp.  The compression is
  * applied at the end of the prefill (Section 4, Figure 4): a caller that computes its prefill attention here hands

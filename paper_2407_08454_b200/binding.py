@@ -24,7 +24,7 @@ KVM_WEIGHT_GAUSSIAN, KVM_WEIGHT_AVERAGE, KVM_WEIGHT_PIVOT_ONLY, KVM_WEIGHT_SET_S
 KVM_SETS_ADJACENT, KVM_SETS_CONSERVED_ONLY, KVM_SETS_ANCHOR = 0, 1, 2
 EXPORTS = (
     "kvm_sizes", "kvm_workspace_bytes", "kvm_score", "kvm_row_lse", "kvm_segment", "kvm_merge_compact", "kvm_compress",
-    "kvm_compress_with_lse",
+    "kvm_compress_with_lse", "kvm_compress_layers",
     "kvm_host_staging_bytes", "kvm_compress_host", "kvm_score_static", "kvm_layer_ratio", "kvm_attend",
     "kvm_output_perturbation", "kvm_prefill_attend", "kvm_status_string",
     "kvm_version",
@@ -263,18 +263,24 @@ class Compressor:
 
 def compress_layers(p: KvmParams, layers, sim_thresholds=None, device="cuda", stream=None):
     """Compress a stack of layers, each an (Q, K, V) triple of CUDA tensors of the shape `p` describes, with one
-    similarity threshold per layer (Section 3.2: thresholds chosen layer by layer).  Returns, per layer, a
-    `Compressed` holding copies of the outputs, and the layer's compression ratio mean(out_len) / S."""
+    similarity threshold per layer (Section 3.2: thresholds chosen layer by layer), through kvm_compress_layers.
+    Returns, per layer, a `Compressed` holding the outputs, and the layer's compression ratio mean(out_len) / S."""
     n = len(layers)
-    if sim_thresholds is None:
-        sim_thresholds = [p.sim_threshold] * n
-    assert len(sim_thresholds) == n
-    out, ratios = [], []
-    for (Q, K, V), eps in zip(layers, sim_thresholds):
-        pl = KvmParams.from_buffer_copy(bytes(p))
-        pl.sim_threshold = float(eps)
-        c = Compressor(pl, device=device)
-        r = c(Q, K, V, stream=stream)
-        out.append(r)
-        ratios.append(r.out_len.float().mean() / p.seq)
-    return out, [float(x) for x in ratios]
+    comps = [Compressor(p, device=device) for _ in range(n)]
+    ptrs = lambda ts: (ctypes.c_void_p * n)(*[t.data_ptr() for t in ts])
+    for Q, K, V in layers:
+        assert Q.is_contiguous() and K.is_contiguous() and V.is_contiguous()
+    eps = None
+    if sim_thresholds is not None:
+        assert len(sim_thresholds) == n
+        eps = (ctypes.c_float * n)(*[float(e) for e in sim_thresholds])
+    ws = comps[0].ws
+    _check(lib().kvm_compress_layers(ctypes.byref(p), ctypes.c_int32(n), eps, ptrs([l[0] for l in layers]),
+                                     ptrs([l[1] for l in layers]), ptrs([l[2] for l in layers]),
+                                     ptrs([c.K_out for c in comps]), ptrs([c.V_out for c in comps]),
+                                     ptrs([c.out_len for c in comps]), ptrs([c.out_pos for c in comps]),
+                                     ctypes.c_void_p(0), _ptr(ws), ctypes.c_size_t(ws.numel()), _stream(stream)),
+           "kvm_compress_layers")
+    out = [Compressed(c.K_out, c.V_out, c.out_len, c.out_pos, None, c.cap) for c in comps]
+    ratios = [float(c.out_len.float().mean() / p.seq) for c in comps]
+    return out, ratios

@@ -346,6 +346,33 @@ int kvm_compress_with_lse(const kvm_params* p, const void* Q, const void* K, con
     return KVM_OK;
 }
 
+int kvm_compress_layers(const kvm_params* p, int32_t n_layers, const float* sim_thresholds, const void* const* Q,
+                        const void* const* K, const void* const* V, void* const* K_out, void* const* V_out,
+                        int32_t* const* out_len, int32_t* const* out_pos, kvm_stats* stats, void* ws,
+                        size_t ws_bytes, void* cuda_stream) {
+    Dims d;
+    int rc = derive(p, d);
+    if (rc != KVM_OK) return rc;
+    if (n_layers < 1) return KVM_E_SHAPE;
+    if (!Q || !K || !V || !K_out || !V_out || !out_len || !out_pos) return KVM_E_NULL;
+    Workspace w;
+    if ((rc = check_ws(d, ws, ws_bytes, w)) != KVM_OK) return rc;
+    for (int32_t l = 0; l < n_layers; ++l) {       // everything is checked before the first layer is enqueued
+        if (!Q[l] || !K[l] || !V[l] || !K_out[l] || !V_out[l] || !out_len[l] || !out_pos[l]) return KVM_E_NULL;
+        if (misaligned(Q[l]) || misaligned(K[l]) || misaligned(V[l]) || misaligned(K_out[l]) || misaligned(V_out[l]))
+            return KVM_E_ALIGN;
+        if (sim_thresholds && !isfinite(sim_thresholds[l])) return KVM_E_PARAM;
+    }
+    for (int32_t l = 0; l < n_layers; ++l) {
+        kvm_params pl = *p;
+        if (sim_thresholds) pl.sim_threshold = sim_thresholds[l];
+        rc = kvm_compress(&pl, Q[l], K[l], V[l], K_out[l], V_out[l], out_len[l], out_pos[l], nullptr, stats, ws,
+                          ws_bytes, cuda_stream);
+        if (rc != KVM_OK) return rc;
+    }
+    return KVM_OK;
+}
+
 int kvm_host_staging_bytes(const kvm_params* p, size_t* bytes) {
     Dims d;
     const int rc = derive(p, d);

@@ -97,6 +97,23 @@ def test_null_alignment_and_workspace_errors(lib):
     assert lib.kvm_score(None, ok, ok, vp(0), ok, ok, ctypes.c_size_t(1 << 30), vp(0)) == -1
 
 
+def test_layer_stack_entry_point_checks_every_layer_before_it_enqueues(lib):
+    p = kvm.make_params(1, 2, 2, 256, 64, kvm.KVM_BF16)
+    vp = ctypes.c_void_p
+    ok2 = (vp * 2)(4096, 4096)
+    bad2 = (vp * 2)(4096, 0)                       # the second layer's pointer is missing
+    off2 = (vp * 2)(4096, 4100)                    # ... or not 16-byte aligned
+    ws, n = vp(4096), ctypes.c_size_t(1 << 30)
+    call = lambda nl, eps, Q: lib.kvm_compress_layers(ctypes.byref(p), ctypes.c_int32(nl), eps, Q, ok2, ok2, ok2, ok2,
+                                                      ok2, ok2, vp(0), ws, n, vp(0))
+    assert call(0, None, ok2) == -2                # KVM_E_SHAPE
+    assert call(2, None, bad2) == -1               # KVM_E_NULL
+    assert call(2, None, off2) == -5               # KVM_E_ALIGN
+    assert call(2, (ctypes.c_float * 2)(0.75, float("nan")), ok2) == -4      # KVM_E_PARAM
+    assert lib.kvm_compress_layers(ctypes.byref(p), ctypes.c_int32(2), None, ok2, ok2, ok2, ok2, ok2, ok2, ok2, vp(0),
+                                   ws, ctypes.c_size_t(16), vp(0)) == -6     # KVM_E_WORKSPACE
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "_lib", None)
     monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "libkvm.so"))
