@@ -36,20 +36,18 @@ template <typename T> __device__ __forceinline__ T f32_to_elem(float v);
 template <> __device__ __forceinline__ float f32_to_elem<float>(float v) { return v; }
 template <> __device__ __forceinline__ __nv_bfloat16 f32_to_elem<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
-// set_id[u][j] = index of the set holding token j, from the sets' start positions.
+// set_id[u][j] = index of the set holding token j, from the sets' start positions: one thread per set writes
+// its index over the set's tokens (sets are a few tokens long on average; a long one costs its thread a loop).
 __global__ void __launch_bounds__(256) token_set_kernel(const int32_t* __restrict__ set_start,
                                                         const int32_t* __restrict__ out_len,
                                                         int32_t* __restrict__ set_id, int S, int cap) {
     const int u = blockIdx.y;
-    const int j = blockIdx.x * blockDim.x + threadIdx.x;
-    if (j >= S) return;
+    const int s = blockIdx.x * blockDim.x + threadIdx.x;
+    if (s >= min(out_len[u], cap)) return;
     const int32_t* st = set_start + (size_t)u * (cap + 1);
-    int lo = 0, hi = min(out_len[u], cap);      // largest s in [0, hi) with st[s] <= j
-    while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if (__ldg(st + mid) <= j) lo = mid; else hi = mid;
-    }
-    set_id[(size_t)u * S + j] = lo;
+    const int beg = __ldg(st + s), end = min(__ldg(st + s + 1), S);
+    int32_t* dst = set_id + (size_t)u * S;
+    for (int j = beg; j < end; ++j) dst[j] = s;
 }
 
 // Scratch layout per (unit, tile): [head | tail] x (2*D sums: K channels then V channels), and 2 weight sums.
@@ -423,7 +421,7 @@ size_t merge_scratch_floats(const Dims& d) {
 
 cudaError_t launch_token_sets(const Dims& d, const int32_t* set_start, const int32_t* out_len, int32_t* set_id,
                               cudaStream_t st) {
-    token_set_kernel<<<dim3((d.S + 255) / 256, d.U), 256, 0, st>>>(set_start, out_len, set_id, d.S, d.cap);
+    token_set_kernel<<<dim3((d.cap + 255) / 256, d.U), 256, 0, st>>>(set_start, out_len, set_id, d.S, d.cap);
     return cudaGetLastError();
 }
 

@@ -43,7 +43,8 @@ def _check(O, lse, refO, ref_lse, V, G):
 
 
 @pytest.mark.parametrize("S,D,Hq,Hkv,B", [(640, 128, 4, 2, 1), (300, 64, 2, 2, 2), (1024, 128, 8, 2, 1), (129, 128, 1, 1, 1),
-                                          (77, 64, 4, 1, 1)])
+                                          (77, 64, 4, 1, 1),
+                                          (1100, 64, 40, 8, 1)])      # 360 work items: several per CTA, ragged last tile
 def test_prefill_attention_matches_the_checker_elementwise(S, D, Hq, Hkv, B):
     from oracle import kvmo
     cfg = si.CONFIGS["C1"].scaled(seq=S, head_dim=D, n_q_heads=Hq, n_kv_heads=Hkv, batch=B, seed=31)
