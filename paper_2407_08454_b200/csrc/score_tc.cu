@@ -384,9 +384,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     }
                 } else {
                     int btile = bt0;
-                    for (int h = 0; h < nh; ++h) {
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        if (h >= nh) break;
                         const bool diag = (btile == tile);
-#pragma unroll 1
+#pragma unroll
                         for (int k = 0; k < QPW; ++k) {
                             const int cq = part * QPW + k;       // column quarter of this chunk within the sub-tile
                             // On the diagonal tile whole quarters are masked (skip) or fully valid.
