@@ -35,16 +35,20 @@ __device__ __forceinline__ uint32_t order_key(float f) {
 }
 
 struct Shared {
-    int hist[256];
-    int warp_i[NW];
+    int hist[3][256];       // radix-select histograms, used in rotation (one block barrier per digit)
+    int warp_i[2][NW];      // per-warp totals of the block scans, two buffers used alternately
     float warp_a[NW];
     int warp_p[NW];
     int warp_f[NW];
-    int bcast[4];
+    int tot[4];             // block-wide counters (hard cuts, soft cuts, near-threshold pairs)
 };
 
+// Block scans with ONE barrier each: every warp leaves its total in shared memory, and after the barrier every
+// warp scans the 32 totals for itself.  Consecutive scans must alternate `buf`: a warp can only reach the scan
+// after next (same buffer) once all warps have passed the barrier in between, i.e. finished reading this one.
+
 // Exclusive prefix sum of one int per thread; returns the block total through `total`.
-__device__ __forceinline__ int block_exscan(int v, int& total, Shared& sh) {
+__device__ __forceinline__ int block_exscan(int v, int& total, Shared& sh, int buf) {
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     int inc = v;
 #pragma unroll
@@ -52,26 +56,21 @@ __device__ __forceinline__ int block_exscan(int v, int& total, Shared& sh) {
         const int t = __shfl_up_sync(0xffffffffu, inc, off);
         if (lane >= off) inc += t;
     }
-    __syncthreads();  // protect warp_i from a previous use
-    if (lane == 31) sh.warp_i[w] = inc;
+    if (lane == 31) sh.warp_i[buf][w] = inc;
     __syncthreads();
-    if (w == 0) {
-        int x = sh.warp_i[lane], xi = x;
+    const int x = sh.warp_i[buf][lane];
+    int xi = x;
 #pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const int t = __shfl_up_sync(0xffffffffu, xi, off);
-            if (lane >= off) xi += t;
-        }
-        sh.warp_i[lane] = xi - x;  // exclusive warp offsets
-        if (lane == 31) sh.bcast[0] = xi;
+    for (int off = 1; off < 32; off <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, xi, off);
+        if (lane >= off) xi += t;
     }
-    __syncthreads();
-    total = sh.bcast[0];
-    return sh.warp_i[w] + inc - v;
+    total = __shfl_sync(0xffffffffu, xi, 31);
+    return __shfl_sync(0xffffffffu, xi - x, w) + inc - v;
 }
 
 // Exclusive prefix maximum of one int per thread (identity -1).
-__device__ __forceinline__ int block_exscan_max(int v, Shared& sh) {
+__device__ __forceinline__ int block_exscan_max(int v, Shared& sh, int buf) {
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     int inc = v;
 #pragma unroll
@@ -79,73 +78,87 @@ __device__ __forceinline__ int block_exscan_max(int v, Shared& sh) {
         const int t = __shfl_up_sync(0xffffffffu, inc, off);
         if (lane >= off) inc = max(inc, t);
     }
-    __syncthreads();  // protect warp_i from a previous use
-    if (lane == 31) sh.warp_i[w] = inc;
+    if (lane == 31) sh.warp_i[buf][w] = inc;
     __syncthreads();
-    if (w == 0) {
-        int x = sh.warp_i[lane];
+    int x = sh.warp_i[buf][lane];
 #pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const int t = __shfl_up_sync(0xffffffffu, x, off);
-            if (lane >= off) x = max(x, t);
-        }
-        const int ex = __shfl_up_sync(0xffffffffu, x, 1);
-        sh.warp_i[lane] = lane ? ex : -1;    // exclusive over warps
+    for (int off = 1; off < 32; off <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, x, off);
+        if (lane >= off) x = max(x, t);
     }
-    __syncthreads();
+    const int before_warp = __shfl_sync(0xffffffffu, x, (w + 31) & 31);   // inclusive maximum over warps 0..w-1
     const int prev = __shfl_up_sync(0xffffffffu, inc, 1);
-    return max(sh.warp_i[w], lane ? prev : -1);
+    return max(w ? before_warp : -1, lane ? prev : -1);
 }
 
-// Among the tokens j in [0, n) for which valid(j), find the k smallest keys (k >= 1,
-// k <= number of valid tokens).  On return every valid token with key < cut is
-// selected, and of those with key == cut the first `need` in index order are.
+// Among the tokens j in [lo, hi) of every thread for which valid(j), find the k smallest keys (k >= 1,
+// k <= number of valid tokens).  On return every valid token with key < cut is selected, and of the `n_eq`
+// tokens with key == cut the first `need` in index order are.
+// Four 8-bit digits, most significant first.  A digit costs one block barrier: the histograms rotate through
+// three buffers (digit p counts into buffer p mod 3 and clears the one digit p + 2 will use, which nobody has
+// read since the barrier before), and every warp finds the digit's bin for itself from the finished histogram
+// instead of waiting for one warp to publish it.
 template <typename KeyFn, typename ValidFn>
-__device__ __forceinline__ void radix_select(int n, int k, KeyFn key, ValidFn valid, uint32_t& cut, int& need,
-                                             Shared& sh) {
+__device__ __forceinline__ void radix_select(int lo, int hi, int k, KeyFn key, ValidFn valid, uint32_t& cut,
+                                             int& need, int& n_eq, Shared& sh) {
+    const int lane = threadIdx.x & 31;
+    if (threadIdx.x < 512) sh.hist[threadIdx.x >> 8][threadIdx.x & 255] = 0;
+    __syncthreads();
     uint32_t prefix = 0, mask = 0;
-    int k_rem = k;
-    for (int shift = 24; shift >= 0; shift -= 8) {
+    int k_rem = k, cnt = 0;
+#pragma unroll
+    for (int p = 0; p < 4; ++p) {
+        const int shift = 24 - 8 * p;
+        int* H = sh.hist[p % 3];
+        // a thread's tokens are neighbours and often share a bin: count runs, one atomic per run
+        int run_bin = -1, run_n = 0;
+        for (int j = lo; j < hi; ++j) {
+            if (!valid(j)) continue;
+            const uint32_t kk = key(j);
+            if ((kk & mask) != prefix) continue;
+            const int bin = (int)((kk >> shift) & 255u);
+            if (bin != run_bin) {
+                if (run_n) atomicAdd(&H[run_bin], run_n);
+                run_bin = bin;
+                run_n = 0;
+            }
+            ++run_n;
+        }
+        if (run_n) atomicAdd(&H[run_bin], run_n);
         __syncthreads();
-        if (threadIdx.x < 256) sh.hist[threadIdx.x] = 0;
-        __syncthreads();
-        for (int j = threadIdx.x; j < n; j += NT) {
-            if (valid(j)) {
-                const uint32_t kk = key(j);
-                if ((kk & mask) == prefix) atomicAdd(&sh.hist[(kk >> shift) & 255u], 1);
+        // lane l owns bins [8l, 8l+8): find the bin where the running count reaches k_rem
+        const int4 c0 = reinterpret_cast<const int4*>(H)[lane * 2], c1 = reinterpret_cast<const int4*>(H)[lane * 2 + 1];
+        const int c[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+        int s = 0;
+#pragma unroll
+        for (int t = 0; t < 8; ++t) s += c[t];
+        int inc = s;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, inc, off);
+            if (lane >= off) inc += t;
+        }
+        int below = inc - s, bin = 0, bin_below = 0, bin_cnt = 0;
+        const bool mine = below < k_rem && k_rem <= inc;       // true in exactly one lane
+        if (mine) {
+#pragma unroll
+            for (int t = 0; t < 8; ++t) {
+                if (below < k_rem && k_rem <= below + c[t]) { bin = lane * 8 + t; bin_below = below; bin_cnt = c[t]; }
+                below += c[t];
             }
         }
-        __syncthreads();
-        if (threadIdx.x < 32) {
-            // lane l owns bins [8l, 8l+8): find the bin where the running count reaches k_rem
-            int c[8], s = 0;
-#pragma unroll
-            for (int t = 0; t < 8; ++t) { c[t] = sh.hist[threadIdx.x * 8 + t]; s += c[t]; }
-            int inc = s;
-#pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                const int t = __shfl_up_sync(0xffffffffu, inc, off);
-                if ((int)threadIdx.x >= off) inc += t;
-            }
-            int below = inc - s;
-            if (below < k_rem && k_rem <= inc) {
-#pragma unroll
-                for (int t = 0; t < 8; ++t) {
-                    if (below < k_rem && k_rem <= below + c[t]) {
-                        sh.bcast[1] = threadIdx.x * 8 + t;
-                        sh.bcast[2] = below;
-                    }
-                    below += c[t];
-                }
-            }
-        }
-        __syncthreads();
-        prefix |= (uint32_t)sh.bcast[1] << shift;
+        const int src = __ffs(__ballot_sync(0xffffffffu, mine)) - 1;
+        bin = __shfl_sync(0xffffffffu, bin, src);
+        bin_below = __shfl_sync(0xffffffffu, bin_below, src);
+        cnt = __shfl_sync(0xffffffffu, bin_cnt, src);
+        prefix |= (uint32_t)bin << shift;
         mask |= 255u << shift;
-        k_rem -= sh.bcast[2];
+        k_rem -= bin_below;
+        if (p < 2 && threadIdx.x < 256) sh.hist[(p + 2) % 3][threadIdx.x] = 0;
     }
     cut = prefix;
     need = k_rem;
+    n_eq = cnt;
 }
 
 struct Best {
@@ -154,6 +167,17 @@ struct Best {
 };
 // Left operand covers lower indices; ties keep the left (lower index).
 __device__ __forceinline__ Best better(Best l, Best r) { return (r.a > l.a) ? r : l; }
+
+__device__ __forceinline__ void record_out_len(kvm_stats* stats, int n) {
+    atomicMax(&stats->max_out_len, n);
+    int old = stats->min_out_len;      // 0 means "unset"
+    while (old == 0 || n < old) {
+        const int prev = atomicCAS(&stats->min_out_len, old, n);
+        if (prev == old) break;
+        old = prev;
+    }
+    atomicAdd((unsigned long long*)&stats->sum_out_len, (unsigned long long)n);
+}
 
 __global__ void __launch_bounds__(NT) segment_unit_kernel(const float* __restrict__ scores,
                                                           const float* __restrict__ sim, int32_t* __restrict__ set_id,
@@ -176,18 +200,25 @@ __global__ void __launch_bounds__(NT) segment_unit_kernel(const float* __restric
     const int R = max(0, S - n_r);                 // first recent position
     const int nh = min(n_h, R);
 
+    if (threadIdx.x < 4) sh.tot[threadIdx.x] = 0;   // (the barriers of step 1 come before their first use)
+
     // ---- 1. conserved set: recent window + n_h largest scores (ties: lower index)
     uint32_t cut = 0;
-    int need = 0;
+    int need = 0, n_eq = 0;
     if (nh > 0) {
-        radix_select(R, nh, [&](int j) { return ~order_key(a[j]); }, [&](int) { return true; }, cut, need, sh);
+        radix_select(lo, min(hi, R), nh, [&](int j) { return ~order_key(a[j]); }, [&](int) { return true; }, cut,
+                     need, n_eq, sh);
     }
     {
-        int eq = 0;
-        if (nh > 0)
+        // Tokens whose key equals the cut are taken in index order until `need` are; when all of them are
+        // needed (no tie at the cut: the usual case) their ranks do not matter and the scan is skipped.
+        int rank = 0;
+        if (nh > 0 && need < n_eq) {
+            int eq = 0;
             for (int j = lo; j < min(hi, R); ++j) eq += (~order_key(a[j]) == cut);
-        int tot;
-        int rank = block_exscan(eq, tot, sh);
+            int tot;
+            rank = block_exscan(eq, tot, sh, 0);
+        }
         for (int j = lo; j < hi; ++j) {
             uint8_t f = 0;
             if (j >= R) f = F_KEEP;
@@ -209,7 +240,7 @@ __global__ void __launch_bounds__(NT) segment_unit_kernel(const float* __restric
         int nk = 0;
         for (int j = lo; j < hi; ++j) nk += (flags[j] & F_KEEP) ? 1 : 0;
         int n_keep;
-        int id = block_exscan(nk, n_keep, sh);
+        int id = block_exscan(nk, n_keep, sh, 1);
         for (int j = lo; j < hi; ++j) {
             const bool k = (flags[j] & F_KEEP) != 0;
             if (k && id < cap) { st[id] = j; pv[id] = j; }
@@ -220,14 +251,7 @@ __global__ void __launch_bounds__(NT) segment_unit_kernel(const float* __restric
             if (n_keep <= cap) st[n_keep] = S;
             out_len[u] = n_keep;
             if (stats) {
-                atomicMax(&stats->max_out_len, n_keep);
-                int old = stats->min_out_len;      // 0 means "unset"
-                while (old == 0 || n_keep < old) {
-                    const int prev = atomicCAS(&stats->min_out_len, old, n_keep);
-                    if (prev == old) break;
-                    old = prev;
-                }
-                atomicAdd((unsigned long long*)&stats->sum_out_len, (unsigned long long)n_keep);
+                record_out_len(stats, n_keep);
             }
         }
         return;
@@ -244,7 +268,7 @@ __global__ void __launch_bounds__(NT) segment_unit_kernel(const float* __restric
         uint16_t* JB = JA + S;
         int last_keep = -1;
         for (int j = lo; j < hi; ++j) if (flags[j] & F_KEEP) last_keep = j;
-        int pk = block_exscan_max(last_keep, sh);            // nearest conserved token before this range
+        int pk = block_exscan_max(last_keep, sh, 1);            // nearest conserved token before this range
         for (int j = lo; j < hi; ++j) {
             const bool kept = (flags[j] & F_KEEP) != 0;
             const int eff = kept ? 0 : min((int)c[j], j - 1 - pk);
@@ -277,25 +301,35 @@ __global__ void __launch_bounds__(NT) segment_unit_kernel(const float* __restric
         else if (!(cj > eps)) { f |= F_SOFT | F_CUT; ++n_soft; }
         flags[j] = f;    // only bits other than F_KEEP change, so neighbours reading F_KEEP are safe
     }
-    int tot_hard, tot_soft;
-    block_exscan(n_hard, tot_hard, sh);
-    block_exscan(n_soft, tot_soft, sh);
-    block_exscan(n_near, tot_near, sh);
+    // block totals: warp sums, one shared-memory atomic per warp and counter (integers: any order gives the same sum)
+    n_hard = __reduce_add_sync(0xffffffffu, n_hard);
+    n_soft = __reduce_add_sync(0xffffffffu, n_soft);
+    n_near = __reduce_add_sync(0xffffffffu, n_near);
+    if ((threadIdx.x & 31) == 0) {
+        if (n_hard) atomicAdd(&sh.tot[0], n_hard);
+        if (n_soft) atomicAdd(&sh.tot[1], n_soft);
+        if (n_near) atomicAdd(&sh.tot[2], n_near);
+    }
+    __syncthreads();
+    const int tot_hard = sh.tot[0], tot_soft = sh.tot[1];
+    tot_near = sh.tot[2];
 
     // ---- 3. budget rule: keep only the (cap - hard) soft cuts with the smallest similarity
     fire = enforce && (tot_hard + tot_soft > cap);
     if (fire) {
         const int m = max(0, cap - tot_hard);
         uint32_t cut2 = 0;
-        int need2 = 0;
+        int need2 = 0, n_eq2 = 0;
         if (m > 0)
-            radix_select(S, m, [&](int j) { return order_key(c[j]); }, [&](int j) { return (flags[j] & F_SOFT) != 0; },
-                         cut2, need2, sh);
-        int eq = 0;
-        if (m > 0)
+            radix_select(lo, hi, m, [&](int j) { return order_key(c[j]); },
+                         [&](int j) { return (flags[j] & F_SOFT) != 0; }, cut2, need2, n_eq2, sh);
+        int rank = 0;
+        if (m > 0 && need2 < n_eq2) {
+            int eq = 0;
             for (int j = lo; j < hi; ++j) eq += ((flags[j] & F_SOFT) && order_key(c[j]) == cut2);
-        int tot;
-        int rank = block_exscan(eq, tot, sh);
+            int tot;
+            rank = block_exscan(eq, tot, sh, 1);
+        }
         for (int j = lo; j < hi; ++j) {
             const uint8_t f = flags[j];
             if (f & F_SOFT) {
@@ -310,13 +344,13 @@ __global__ void __launch_bounds__(NT) segment_unit_kernel(const float* __restric
         }
     }
     }   // neighbour reading
-    __syncthreads();
+    // (no barrier: from here on a thread reads only the flags of its own tokens, which it wrote itself)
 
     // ---- 4. scan of the cut flags -> set ids and starts
     int ncut = 0;
     for (int j = lo; j < hi; ++j) ncut += (flags[j] & F_CUT) ? 1 : 0;
     int n_sets;
-    const int before = block_exscan(ncut, n_sets, sh);
+    const int before = block_exscan(ncut, n_sets, sh, 0);
     {
         int id = before - 1;
         for (int j = lo; j < hi; ++j) {
@@ -333,14 +367,7 @@ __global__ void __launch_bounds__(NT) segment_unit_kernel(const float* __restric
         if (stats) {
             if (fire) atomicAdd(&stats->units_budget_rule, 1);
             if (tot_near) atomicAdd(&stats->near_threshold, tot_near);
-            atomicMax(&stats->max_out_len, n_sets);
-            int old = stats->min_out_len;      // 0 means "unset"
-            while (old == 0 || n_sets < old) {
-                const int prev = atomicCAS(&stats->min_out_len, old, n_sets);
-                if (prev == old) break;
-                old = prev;
-            }
-            atomicAdd((unsigned long long*)&stats->sum_out_len, (unsigned long long)n_sets);
+            record_out_len(stats, n_sets);
         }
     }
 
@@ -378,31 +405,25 @@ __global__ void __launch_bounds__(NT) segment_unit_kernel(const float* __restric
         const int lf = __shfl_up_sync(0xffffffffu, xf, off);
         if (lane >= off && !xf) { x = better(Best{la, li}, x); xf = lf; }
     }
-    __syncthreads();
     if (lane == 31) { sh.warp_a[w] = x.a; sh.warp_p[w] = x.i; sh.warp_f[w] = xf; }
     __syncthreads();
-    if (w == 0) {
-        Best y = {sh.warp_a[lane], sh.warp_p[lane]};
-        int yf = sh.warp_f[lane];
+    // every warp scans the 32 warp aggregates for itself; the carry into warp w is the inclusive value of warp w-1
+    Best y = {sh.warp_a[lane], sh.warp_p[lane]};
+    int yf = sh.warp_f[lane];
 #pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const float la = __shfl_up_sync(0xffffffffu, y.a, off);
-            const int li = __shfl_up_sync(0xffffffffu, y.i, off);
-            const int lf = __shfl_up_sync(0xffffffffu, yf, off);
-            if (lane >= off && !yf) { y = better(Best{la, li}, y); yf = lf; }
-        }
-        // exclusive: shift by one warp
-        const float ea = __shfl_up_sync(0xffffffffu, y.a, 1);
-        const int ei = __shfl_up_sync(0xffffffffu, y.i, 1);
-        sh.warp_a[lane] = lane ? ea : -INFINITY;
-        sh.warp_p[lane] = lane ? ei : INT_MAX;
+    for (int off = 1; off < 32; off <<= 1) {
+        const float la = __shfl_up_sync(0xffffffffu, y.a, off);
+        const int li = __shfl_up_sync(0xffffffffu, y.i, off);
+        const int lf = __shfl_up_sync(0xffffffffu, yf, off);
+        if (lane >= off && !yf) { y = better(Best{la, li}, y); yf = lf; }
     }
-    __syncthreads();
+    const float wa = __shfl_sync(0xffffffffu, y.a, (w + 31) & 31);
+    const int wi = __shfl_sync(0xffffffffu, y.i, (w + 31) & 31);
     // carry into this thread = (carry into its warp) (+) (inclusive value of the previous lane)
     const float pa = __shfl_up_sync(0xffffffffu, x.a, 1);
     const int pi = __shfl_up_sync(0xffffffffu, x.i, 1);
     const int pf = __shfl_up_sync(0xffffffffu, xf, 1);
-    Best carry = {sh.warp_a[w], sh.warp_p[w]};
+    Best carry = w ? Best{wa, wi} : Best{-INFINITY, INT_MAX};
     if (lane > 0) carry = pf ? Best{pa, pi} : better(carry, Best{pa, pi});
     // The set that was open when this thread's range began ends at its first cut
     // (or at the end of the sequence, for the thread holding the last token).
@@ -412,6 +433,333 @@ __global__ void __launch_bounds__(NT) segment_unit_kernel(const float* __restric
             if (ended >= 0 && ended < cap) pv[ended] = better(carry, head).i;
             if (hi == S && id < cap) pv[id] = run.i;
         } else if (hi == S) {
+            if (id >= 0 && id < cap) pv[id] = better(carry, head).i;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// The same step for the neighbour reading when a thread's share is at most EM tokens (S <= EM * 1024): scores,
+// similarities, keys and flags stay in registers, every token loop is unrolled, and neighbouring threads
+// exchange the one bit they need by shuffle.  With 32 warps on one SM the kernel is bound by instruction issue,
+// so what counts is instructions per token; results are identical to segment_unit_kernel's.
+struct SharedReg {
+    int hist[3][2048];      // one histogram per digit of the radix select
+    int warp_i[2][NW];      // per-warp totals of the block scans, two buffers used alternately
+    float warp_a[NW];
+    int warp_p[NW];
+    int warp_f[NW];
+    int tot[4];             // block-wide counters (hard cuts, soft cuts, near-threshold pairs)
+    int found[3][4];        // per digit: bin, keys below it, keys in it
+};
+
+// Exclusive prefix sum of one int per thread with one barrier (see block_exscan above for the two buffers).
+__device__ __forceinline__ int block_exscan(int v, int& total, SharedReg& sh, int buf) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    int inc = v;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, inc, off);
+        if (lane >= off) inc += t;
+    }
+    if (lane == 31) sh.warp_i[buf][w] = inc;
+    __syncthreads();
+    const int x = sh.warp_i[buf][lane];
+    int xi = x;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, xi, off);
+        if (lane >= off) xi += t;
+    }
+    total = __shfl_sync(0xffffffffu, xi, 31);
+    return __shfl_sync(0xffffffffu, xi - x, w) + inc - v;
+}
+
+// The k smallest of the keys marked in `valid` (bit t = key[t]); results as radix_select's.  Three digits of
+// 11, 11 and 10 bits: the block's 1024 threads own two bins each, a block scan over the bin counts finds the
+// digit, and the one thread whose bins hold the k-th key publishes it.  (Eight-bit digits with every warp
+// scanning 256 bins for itself cost more instructions in total, and instruction issue is what bounds this kernel.)
+template <int EM>
+__device__ __forceinline__ void radix_select_reg(const uint32_t (&key)[EM], unsigned valid, int k, uint32_t& cut,
+                                                 int& need, int& n_eq, SharedReg& sh) {
+    static_assert(NT == 1024, "two bins per thread");
+    {
+        int* h = &sh.hist[0][0];
+#pragma unroll
+        for (int i = 0; i < 6; ++i) h[i * NT + threadIdx.x] = 0;
+    }
+    __syncthreads();
+    uint32_t prefix = 0, mask = 0;
+    int k_rem = k, cnt = 0;
+#pragma unroll
+    for (int p = 0; p < 3; ++p) {
+        const int shift = p == 0 ? 21 : (p == 1 ? 10 : 0);
+        const uint32_t dmask = p == 2 ? 1023u : 2047u;
+        int* H = sh.hist[p];
+        if (p == 0) {
+            // the leading digit of neighbouring tokens is often the same: one atomic per run
+            int run_bin = -1, run_n = 0;
+#pragma unroll
+            for (int t = 0; t < EM; ++t) {
+                if (!((valid >> t) & 1u)) continue;
+                const int bin = (int)(key[t] >> 21);
+                if (bin != run_bin) {
+                    if (run_n) atomicAdd(&H[run_bin], run_n);
+                    run_bin = bin;
+                    run_n = 0;
+                }
+                ++run_n;
+            }
+            if (run_n) atomicAdd(&H[run_bin], run_n);
+        } else {
+#pragma unroll
+            for (int t = 0; t < EM; ++t)
+                if (((valid >> t) & 1u) && (key[t] & mask) == prefix) atomicAdd(&H[(key[t] >> shift) & dmask], 1);
+        }
+        __syncthreads();
+        const int2 h = reinterpret_cast<const int2*>(H)[threadIdx.x];     // bins 2t, 2t+1
+        const int s = h.x + h.y;
+        int tot;
+        const int below = block_exscan(s, tot, sh, p & 1);
+        if (below < k_rem && k_rem <= below + s) {                        // true in exactly one thread
+            const bool first = k_rem <= below + h.x;
+            sh.found[p][0] = 2 * (int)threadIdx.x + (first ? 0 : 1);
+            sh.found[p][1] = first ? below : below + h.x;
+            sh.found[p][2] = first ? h.x : h.y;
+        }
+        __syncthreads();
+        prefix |= (uint32_t)sh.found[p][0] << shift;
+        mask |= dmask << shift;
+        k_rem -= sh.found[p][1];
+        cnt = sh.found[p][2];
+    }
+    cut = prefix;
+    need = k_rem;
+    n_eq = cnt;
+}
+
+template <int EM>
+__global__ void __launch_bounds__(NT) segment_unit_reg_kernel(const float* __restrict__ scores,
+                                                              const float* __restrict__ sim,
+                                                              int32_t* __restrict__ set_id,
+                                                              int32_t* __restrict__ set_start,
+                                                              int32_t* __restrict__ pivot, int32_t* __restrict__ out_len,
+                                                              kvm_stats* stats, int S, int cap, int n_r, int n_h,
+                                                              float eps, int enforce, int pivot_rule,
+                                                              const float* __restrict__ pivot_key) {
+    __shared__ SharedReg sh;
+    grid_launch_dependents();   // (as in segment_unit_kernel)
+    grid_dependency_wait();
+    const int u = blockIdx.x;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int E = (S + NT - 1) / NT;               // tokens per thread, contiguous; E <= EM
+    const int lo = min(S, (int)threadIdx.x * E);
+    const int n = min(E, S - lo);                  // this thread's tokens: lo .. lo+n-1
+    const int R = max(0, S - n_r);                 // first recent position
+    const int nh = min(n_h, R);
+    if (threadIdx.x < 4) sh.tot[threadIdx.x] = 0;  // (barriers of step 1 come before their first use)
+
+    float a[EM], c[EM];
+    uint32_t ka[EM];
+    const size_t g0 = (size_t)u * S + lo;          // this thread's first token in the [U, S] arrays
+    const bool vec = EM == 4 && n == 4 && (g0 & 3) == 0;   // four tokens on a 16-byte boundary: one access per array
+    if (vec) {
+        const float4 av = *reinterpret_cast<const float4*>(scores + g0), cv = *reinterpret_cast<const float4*>(sim + g0);
+        a[0] = av.x; a[1] = av.y; a[2] = av.z; a[3] = av.w;
+        c[0] = cv.x; c[1] = cv.y; c[2] = cv.z; c[3] = cv.w;
+    } else {
+#pragma unroll
+        for (int t = 0; t < EM; ++t) {
+            a[t] = (t < n) ? scores[g0 + t] : 0.f;
+            c[t] = (t < n) ? sim[g0 + t] : 0.f;
+        }
+    }
+#pragma unroll
+    for (int t = 0; t < EM; ++t) ka[t] = ~order_key(a[t]);
+    const unsigned own = (1u << n) - 1u;                                      // bit t: token lo+t exists
+    const unsigned old_m = own & ((1u << max(0, min(n, R - lo))) - 1u);        // ... and lies before the recent window
+
+    // ---- 1. conserved set: recent window + n_h largest scores (ties: lower index)
+    uint32_t cut = 0;
+    int need = 0, n_eq = 0;
+    if (nh > 0) radix_select_reg<EM>(ka, old_m, nh, cut, need, n_eq, sh);
+    unsigned keep = own & ~old_m;                                             // the recent window
+    if (nh > 0) {
+        int rank = 0;
+        if (need < n_eq) {        // a tie at the cut: the first `need` of the equal keys in index order
+            int eq = 0;
+#pragma unroll
+            for (int t = 0; t < EM; ++t) eq += (((old_m >> t) & 1u) && ka[t] == cut);
+            int tot;
+            rank = block_exscan(eq, tot, sh, 0);
+        } else {
+            rank = INT_MIN;       // every equal key is taken
+        }
+#pragma unroll
+        for (int t = 0; t < EM; ++t) {
+            if (!((old_m >> t) & 1u)) continue;
+            if (ka[t] < cut) keep |= 1u << t;
+            else if (ka[t] == cut) { if (rank < need) keep |= 1u << t; ++rank; }
+        }
+    }
+    // the token before this thread's first: the last token of the thread before (which has all E of its tokens)
+    const unsigned last_keep = (keep >> (E - 1)) & 1u;
+    if (lane == 31) sh.warp_f[w] = (int)last_keep;
+    __syncthreads();
+    unsigned prev_keep = __shfl_up_sync(0xffffffffu, last_keep, 1);
+    if (lane == 0) prev_keep = w ? (unsigned)sh.warp_f[w - 1] : 0u;
+
+    // ---- 2. boundary flags
+    unsigned hardm = 0, softm = 0;
+    int n_near = 0;
+#pragma unroll
+    for (int t = 0; t < EM; ++t) {
+        if (!((own >> t) & 1u)) continue;
+        const int j = lo + t;
+        const unsigned before = t ? (keep >> (t - 1)) & 1u : prev_keep;
+        const bool hard = (j == 0) || ((keep >> t) & 1u) || before;
+        if (j > 0 && fabsf(c[t] - eps) < 1e-3f) ++n_near;
+        if (hard) hardm |= 1u << t;
+        else if (!(c[t] > eps)) softm |= 1u << t;
+    }
+    {
+        const int wh = __reduce_add_sync(0xffffffffu, __popc(hardm));
+        const int ws = __reduce_add_sync(0xffffffffu, __popc(softm));
+        const int wn = __reduce_add_sync(0xffffffffu, n_near);
+        if (lane == 0) {
+            if (wh) atomicAdd(&sh.tot[0], wh);
+            if (ws) atomicAdd(&sh.tot[1], ws);
+            if (wn) atomicAdd(&sh.tot[2], wn);
+        }
+    }
+    __syncthreads();
+    const int tot_hard = sh.tot[0], tot_soft = sh.tot[1], tot_near = sh.tot[2];
+
+    // ---- 3. budget rule: keep only the (cap - hard) soft cuts with the smallest similarity
+    const bool fire = enforce && (tot_hard + tot_soft > cap);
+    unsigned cutm = hardm | softm;
+    if (fire) {
+        const int m = max(0, cap - tot_hard);
+        unsigned stay = 0;
+        if (m > 0) {
+            uint32_t kc[EM];
+#pragma unroll
+            for (int t = 0; t < EM; ++t) kc[t] = order_key(c[t]);
+            uint32_t cut2 = 0;
+            int need2 = 0, n_eq2 = 0;
+            radix_select_reg<EM>(kc, softm, m, cut2, need2, n_eq2, sh);
+            int rank = INT_MIN;
+            if (need2 < n_eq2) {
+                int eq = 0;
+#pragma unroll
+                for (int t = 0; t < EM; ++t) eq += (((softm >> t) & 1u) && kc[t] == cut2);
+                int tot;
+                rank = block_exscan(eq, tot, sh, 1);
+            }
+#pragma unroll
+            for (int t = 0; t < EM; ++t) {
+                if (!((softm >> t) & 1u)) continue;
+                if (kc[t] < cut2) stay |= 1u << t;
+                else if (kc[t] == cut2) { if (rank < need2) stay |= 1u << t; ++rank; }
+            }
+        }
+        cutm = hardm | stay;
+    }
+
+    // ---- 4. scan of the cut flags -> set ids and starts
+    int32_t* st = set_start + (size_t)u * (cap + 1);
+    int32_t* pv = pivot + (size_t)u * cap;
+    int n_sets;
+    const int before = block_exscan(__popc(cutm), n_sets, sh, 0);
+    {
+        int id = before - 1, ids[EM];
+#pragma unroll
+        for (int t = 0; t < EM; ++t) {
+            if (((own & cutm) >> t) & 1u) {
+                ++id;
+                if (id <= cap) st[id] = lo + t;
+            }
+            ids[t] = id;
+        }
+        if (set_id) {
+            if (vec) {
+                *reinterpret_cast<int4*>(set_id + g0) = make_int4(ids[0], ids[1], ids[2], ids[3]);
+            } else {
+#pragma unroll
+                for (int t = 0; t < EM; ++t)
+                    if (t < n) set_id[g0 + t] = ids[t];
+            }
+        }
+    }
+    if (threadIdx.x == 0) {
+        if (n_sets <= cap) st[n_sets] = S;
+        out_len[u] = n_sets;
+        if (stats) {
+            if (fire) atomicAdd(&stats->units_budget_rule, 1);
+            if (tot_near) atomicAdd(&stats->near_threshold, tot_near);
+            record_out_len(stats, n_sets);
+        }
+    }
+
+    // ---- 5. segmented arg-max: pivot of each set (ties: lowest index), as in segment_unit_kernel
+    float key[EM];
+#pragma unroll
+    for (int t = 0; t < EM; ++t) {
+        key[t] = a[t];
+        if (pivot_rule == KVM_PIVOT_LAST) key[t] = (float)(lo + t);
+        else if (pivot_rule == KVM_PIVOT_KEY && t < n) key[t] = pivot_key[g0 + t];
+    }
+    Best head = {-INFINITY, INT_MAX}, run = {-INFINITY, INT_MAX};
+    bool seen_cut = false;
+    int id = before - 1;          // set of the token before `lo`
+    int first_cut_id = -1;        // id of the set that starts at this thread's first cut
+#pragma unroll
+    for (int t = 0; t < EM; ++t) {
+        if (!((own >> t) & 1u)) continue;
+        if ((cutm >> t) & 1u) {
+            if (seen_cut) { if (id < cap) pv[id] = run.i; }       // a set fully inside this range
+            else { head = run; first_cut_id = id + 1; }
+            seen_cut = true;
+            ++id;
+            run = {-INFINITY, INT_MAX};
+        }
+        run = better(run, Best{key[t], lo + t});
+    }
+    if (!seen_cut) head = run;
+    Best x = run;                 // tail if seen_cut, else the whole range (== head)
+    int xf = seen_cut ? 1 : 0;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const float la = __shfl_up_sync(0xffffffffu, x.a, off);
+        const int li = __shfl_up_sync(0xffffffffu, x.i, off);
+        const int lf = __shfl_up_sync(0xffffffffu, xf, off);
+        if (lane >= off && !xf) { x = better(Best{la, li}, x); xf = lf; }
+    }
+    if (lane == 31) { sh.warp_a[w] = x.a; sh.warp_p[w] = x.i; sh.warp_f[w] = xf; }
+    __syncthreads();
+    Best y = {sh.warp_a[lane], sh.warp_p[lane]};
+    int yf = sh.warp_f[lane];
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const float la = __shfl_up_sync(0xffffffffu, y.a, off);
+        const int li = __shfl_up_sync(0xffffffffu, y.i, off);
+        const int lf = __shfl_up_sync(0xffffffffu, yf, off);
+        if (lane >= off && !yf) { y = better(Best{la, li}, y); yf = lf; }
+    }
+    const float wa = __shfl_sync(0xffffffffu, y.a, (w + 31) & 31);
+    const int wi = __shfl_sync(0xffffffffu, y.i, (w + 31) & 31);
+    const float pa = __shfl_up_sync(0xffffffffu, x.a, 1);
+    const int pi = __shfl_up_sync(0xffffffffu, x.i, 1);
+    const int pf = __shfl_up_sync(0xffffffffu, xf, 1);
+    Best carry = w ? Best{wa, wi} : Best{-INFINITY, INT_MAX};
+    if (lane > 0) carry = pf ? Best{pa, pi} : better(carry, Best{pa, pi});
+    if (n > 0) {
+        const bool last = (lo + n == S);
+        if (seen_cut) {
+            const int ended = first_cut_id - 1;
+            if (ended >= 0 && ended < cap) pv[ended] = better(carry, head).i;
+            if (last && id < cap) pv[id] = run.i;
+        } else if (last) {
             if (id >= 0 && id < cap) pv[id] = better(carry, head).i;
         }
     }
@@ -458,6 +806,10 @@ cudaError_t launch_segment(const Dims& d, const float* scores, const float* sim,
                                              (int)segment_max_smem());
         if (e != cudaSuccess) return e;
     }
+    if (d.set_rule == KVM_SETS_ADJACENT && d.S <= 4 * NT)
+        return launch_dependent(segment_unit_reg_kernel<4>, dim3(d.U), dim3(NT), 0, st, scores, sim, set_id, set_start,
+                                pivot, out_len, stats, d.S, d.cap, d.n_r, d.n_h, d.eps, d.enforce, d.pivot_rule,
+                                d.pivot_rule == KVM_PIVOT_KEY ? d.pivot_key : (const float*)nullptr);
     return launch_dependent(segment_unit_kernel, dim3(d.U), dim3(NT), smem, st, scores, sim, set_id, set_start, pivot,
                             out_len, stats, d.S, d.cap, d.n_r, d.n_h, d.eps, d.enforce, d.pivot_rule,
                             d.pivot_rule == KVM_PIVOT_KEY ? d.pivot_key : (const float*)nullptr, d.set_rule);
