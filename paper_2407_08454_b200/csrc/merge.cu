@@ -109,6 +109,9 @@ __global__ void __launch_bounds__(2 * D) merge_tile_kernel(const T* __restrict__
     }
     // The K and V rows are inputs; everything read from here on comes from the kernel before this one.
     grid_dependency_wait();
+    // The fix-up kernel may move in beside this grid's last blocks and look up its sets (written before this
+    // kernel began, as the wait above has just established); it waits for this grid before it reads a slot.
+    grid_launch_dependents();
     {
         // ---- set data per token and the pieces of the tile, while the rows are in flight
         {
@@ -258,23 +261,26 @@ __global__ void __launch_bounds__(2 * D) merge_fixup_kernel(const int32_t* __res
                                                             T* __restrict__ K_out, T* __restrict__ V_out,
                                                             int32_t* __restrict__ out_size, Slots<D> slots, int S,
                                                             int cap, int Tn, int scale_v) {
-    grid_dependency_wait();     // the tile kernel's slots
+    // The sets were written before the tile kernel began (it triggers this launch only after it has waited for
+    // them), so they can be looked up while that kernel's last blocks still run; they are read through L2.
     const int c = blockIdx.x + 1;                 // boundary between tiles c-1 and c
     const long long u = blockIdx.y;
     const int b = c * TOK;
     if (b >= S) return;
     const int32_t* sid_u = set_id + (size_t)u * S;
-    const int sid = sid_u[b];
-    if (sid_u[b - 1] != sid) return;              // no set crosses here
+    const int sid = __ldcg(sid_u + b);
+    if (__ldcg(sid_u + b - 1) != sid) return;     // no set crosses here
     const int32_t* st = set_start + (size_t)u * (cap + 1);
-    const int beg = st[sid], end = st[sid + 1];
+    const int beg = __ldcg(st + sid), end = __ldcg(st + sid + 1);
     if (end > b + TOK) return;                    // crosses a later boundary too: finished there
     const int c_first = beg / TOK;                // tile holding the set's first token (its tail slot)
-    float acc = slots.s(u, Tn, c_first, 1)[threadIdx.x];
-    float gs = *slots.g(u, Tn, c_first, 1);
+    grid_dependency_wait();                       // the tile kernel's slots
+    // (written while this block may already have been resident: read through L2)
+    float acc = __ldcg(slots.s(u, Tn, c_first, 1) + threadIdx.x);
+    float gs = __ldcg(slots.g(u, Tn, c_first, 1));
     for (int t = c_first + 1; t <= c; ++t) {
-        acc += slots.s(u, Tn, t, 0)[threadIdx.x];
-        gs += *slots.g(u, Tn, t, 0);
+        acc += __ldcg(slots.s(u, Tn, t, 0) + threadIdx.x);
+        gs += __ldcg(slots.g(u, Tn, t, 0));
     }
     const int which = threadIdx.x / D, ch = threadIdx.x % D;
     const int n = end - beg;
