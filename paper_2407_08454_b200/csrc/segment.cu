@@ -16,6 +16,10 @@
 // pointer jumping in shared memory.
 // Every tie is broken toward the lower token index, and every reduction has a
 // fixed order, so the integer outputs are reproducible bit for bit.
+// Two kernels compute the same thing: segment_unit_kernel for every shape and
+// rule (tokens re-read per phase, flags in shared memory, 8-bit radix digits),
+// and segment_unit_reg_kernel for the neighbour reading with at most four
+// tokens per thread (S <= 4096), which keeps a thread's tokens in registers.
 #include <limits.h>
 
 #include "common.cuh"

@@ -45,6 +45,35 @@ def test_budget_rule_fires_and_is_exact():
     check_case(case, g)
 
 
+@pytest.mark.parametrize("S", [700, 4101])
+def test_budget_rule_chooses_among_tied_similarities(S):
+    """Zero keys: every similarity is 0 by convention, so every token outside the conserved ones is a cut and the
+    budget rule has to choose among equal keys: the first ones in index order stay.  The short sequence takes the
+    register-resident segment kernel, the long one (more than four tokens per thread) the general one."""
+    g = torch.Generator().manual_seed(40 + S)
+    case = Case(torch.randn(1, 1, S, 64, generator=g), torch.zeros(1, 1, S, 64), torch.randn(1, 1, S, 64, generator=g),
+                budget=0.5, recent=0.05, heavy=0.05, eps=0.5, enforce=True)
+    r = run_gpu(case)
+    assert r.stats.units_budget_rule == 1
+    assert (r.out_len == r.cap).all()
+    check_case(case, r)
+
+
+def test_budget_rule_fires_on_a_sequence_beyond_the_register_kernel():
+    # as test_budget_rule_fires_and_is_exact, on the general segment kernel (S > 4096), with keyed pivots
+    cfg = si.CONFIGS["C1"].scaled(seq=4500, n_q_heads=2, n_kv_heads=2, rho=0.6, budget=0.35, seed=9)
+    case = _case(cfg)
+    case.pivot_rule = kvm.KVM_PIVOT_KEY
+    case.pivot_key = torch.rand((1, 2, 4500), generator=torch.Generator().manual_seed(10), dtype=torch.float32)
+    g = run_gpu(case)
+    assert g.stats.units_budget_rule == 2
+    assert (g.out_len == g.cap).all()
+    check_case(case, g)
+    case = _case(cfg)
+    case.pivot_rule, case.weight_rule = kvm.KVM_PIVOT_LAST, kvm.KVM_WEIGHT_AVERAGE
+    check_case(case)
+
+
 def test_threshold_above_one_returns_the_input_cache():
     cfg = si.CONFIGS["C1"].scaled(seq=512, n_q_heads=2, n_kv_heads=2, seed=8)
     d = si.make_layer(cfg)
