@@ -164,8 +164,12 @@ struct alignas(16) Shared {
     Barriers bar;
     uint32_t tmem_base;
     int abort_flag;
-    float part_m[2][3][TILE];    // row states of warp sets 1..3 at item end, double-buffered by item parity
-    float part_l[2][3][TILE];
+    // Row states of the four warp sets at item end, in three buffers used in rotation (item n uses n mod 3:
+    // the warps that share rows are never three items apart, see the item end), and how many of the four
+    // warps that own a lane quarter's rows have delivered theirs.
+    float part_m[3][4][TILE];
+    float part_l[3][4][TILE];
+    int arrived[3][4];
 };
 
 template <int KCH, int PASS>
@@ -200,6 +204,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         for (int i = 0; i < NSTAGE; ++i) { mbar_init(&sh.bar.full_b[i], 1); mbar_init(&sh.bar.empty_b[i], 1); }
         for (int i = 0; i < NACC; ++i) { mbar_init(&sh.bar.acc_full[i], 1); mbar_init(&sh.bar.acc_empty[i], NEPI_WARPS / 2); }
         sh.abort_flag = 0;
+        for (int i = 0; i < 12; ++i) (&sh.arrived[0][0])[i] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (pass == 2 && threadIdx.x < PTILE_BYTES / 16) {
@@ -428,25 +433,41 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 }
                 ++own;
             }
-            // ---- item end: combine the four partial states of every row (fixed order) and store
-            const int slot = n & 1;
+            // ---- item end: the four warps that own a row (2 groups x 2 column halves) each leave their partial
+            // state in shared memory; whichever of them comes last combines the four in a fixed order (so the
+            // result does not depend on who does it) and stores.  Nobody waits: the group that had the item's
+            // last step is a step behind the other one, which goes straight on to the next item.
+            // (Buffers: a warp is at most one step ahead of a warp of the other group, because the MMA thread
+            // needs the slower group's accumulator back before it can issue the step after next; three items
+            // are at least three steps, so the buffer of item n - 3 has been combined when item n's is written.)
+            const int slot = n % 3;
             const float mine = (pass == 1) ? l : ((acc[0] + acc[1]) + (acc[2] + acc[3])) + ((acc[4] + acc[5]) + (acc[6] + acc[7]));
             constexpr int NPART = NEPI_WARPS / 4;            // partial states per row (one per warp that owns it)
-            if (pidx > 0) { sh.part_m[slot][pidx - 1][row] = m; sh.part_l[slot][pidx - 1][row] = mine; }
-            named_bar(5, NEPI_WARPS * 32);
-            // (read after the barrier: a warp that had no step left when another warp's wait ran out must still
-            // see the flag, or it would store sums that lack the abandoned steps)
-            const bool bad = (*abort_flag != 0);
-            if (pidx == 0) {
+            static_assert(NPART == 4, "four warps own a row");
+            sh.part_m[slot][pidx][row] = m;
+            sh.part_l[slot][pidx][row] = mine;
+            __syncwarp();
+            int before = 0;
+            if (lane == 0) {
+                __threadfence_block();
+                before = atomicAdd(&sh.arrived[slot][lq], 1);
+            }
+            before = __shfl_sync(0xffffffffu, before, 0);
+            if (before == NPART - 1) {
+                __threadfence_block();
+                if (lane == 0) sh.arrived[slot][lq] = 0;     // for item n + 3
+                // (read after all four have delivered: a warp whose wait ran out raised the flag before it came here)
+                const bool bad = (*abort_flag != 0);
                 const int gi = tile * TILE + row;
                 if (gi < S) {
                     if (pass == 1) {
-                        float M = m;
+                        const float m0 = sh.part_m[slot][0][row];
+                        float M = m0;
 #pragma unroll
-                        for (int q = 0; q < NPART - 1; ++q) M = fmaxf(M, sh.part_m[slot][q][row]);
-                        float L = (m > -INFINITY) ? l * ex2(m - M) : 0.f;
+                        for (int q = 1; q < NPART; ++q) M = fmaxf(M, sh.part_m[slot][q][row]);
+                        float L = (m0 > -INFINITY) ? sh.part_l[slot][0][row] * ex2(m0 - M) : 0.f;
 #pragma unroll
-                        for (int q = 0; q < NPART - 1; ++q) {
+                        for (int q = 1; q < NPART; ++q) {
                             const float mq = sh.part_m[slot][q][row], lq_ = sh.part_l[slot][q][row];
                             if (mq > -INFINITY) L += lq_ * ex2(mq - M);
                         }
@@ -461,9 +482,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                                             (uint32_t)__bfloat16_as_ushort(el), 0u, 0u);
                         dst[1] = make_uint4(0u, 0u, 0u, 0u);
                     } else {
-                        float tot = mine;
+                        float tot = sh.part_l[slot][0][row];
 #pragma unroll
-                        for (int q = 0; q < NPART - 1; ++q) tot += sh.part_l[slot][q][row];
+                        for (int q = 1; q < NPART; ++q) tot += sh.part_l[slot][q][row];
                         scores[(size_t)head * S + gi] = bad ? NAN : tot / (float)G;
                     }
                 }
