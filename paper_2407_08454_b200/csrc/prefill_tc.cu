@@ -60,11 +60,14 @@ struct alignas(16) Shared {
 
 struct Sched {
     int P, c, NH, T;
+    // (32-bit arithmetic: the launcher refuses shapes whose item count does not fit; a 64-bit division here costs
+    // every role several hundred clocks at every item boundary)
     __device__ __forceinline__ bool item(int n, int& head, int& tile) const {
-        const long long k = (long long)n * P + ((n & 1) ? (P - 1 - c) : c);
-        if (k >= (long long)NH * T) return false;
-        head = (int)(k % NH);
-        tile = T - 1 - (int)(k / NH);
+        const unsigned k = (unsigned)n * (unsigned)P + (unsigned)((n & 1) ? (P - 1 - c) : c);
+        if (k >= (unsigned)NH * (unsigned)T) return false;
+        const unsigned r = k / (unsigned)NH;
+        head = (int)(k - r * (unsigned)NH);
+        tile = T - 1 - (int)r;
         return true;
     }
 };
@@ -405,6 +408,7 @@ cudaError_t launch_t(const Dims& d, const CUtensorMap& mq, const CUtensorMap& mk
     }
     const int T = (d.S + TILE - 1) / TILE;
     const long long items = (long long)d.B * d.Hq * T;
+    if (items + sms >= (1ll << 31)) return cudaErrorInvalidValue;   // the schedule counts items in 32 bits
     const int grid = (int)(items < sms ? items : sms);
     prefill_attend_kernel<KCH><<<grid, NTHREADS, smem, st>>>(mq, mk, mv, O, lse, stats, d.B, d.Hq, d.Hkv, d.S,
                                                             d.scale * LOG2E);

@@ -118,12 +118,14 @@ struct Sched {
     int P, c, NH, T, G, pass;
     // n-th item of this CTA -> (head or unit, tile).  Items are sorted by descending length
     // (pass 1: query tile T-1 first; pass 2: key tile 0 first) and dealt boustrophedon.
+    // (32-bit arithmetic: NH * T + P stays far below 2^31 for any tensors that fit a GPU, and the launcher
+    // refuses the rest; a 64-bit division here costs every role several hundred clocks at every item boundary)
     __device__ __forceinline__ bool item(int n, int& head, int& tile) const {
-        const long long k = (long long)n * P + ((n & 1) ? (P - 1 - c) : c);
-        if (k >= (long long)NH * T) return false;
-        const int r = (int)(k / NH);
-        head = (int)(k % NH);
-        tile = (pass == 1) ? (T - 1 - r) : r;
+        const unsigned k = (unsigned)n * (unsigned)P + (unsigned)((n & 1) ? (P - 1 - c) : c);
+        if (k >= (unsigned)NH * (unsigned)T) return false;
+        const unsigned r = k / (unsigned)NH;
+        head = (int)(k - r * (unsigned)NH);
+        tile = (pass == 1) ? (T - 1 - (int)r) : (int)r;
         return true;
     }
     __device__ __forceinline__ int ntiles(int tile) const { return (pass == 1) ? tile + 1 : G * (T - tile); }
@@ -568,6 +570,7 @@ cudaError_t launch_t(const Dims& d, const CUtensorMap& mq, const CUtensorMap& mk
     }
     const int T = (d.S + TILE - 1) / TILE;
     const float scale2 = d.scale * LOG2E;
+    if ((long long)d.B * d.Hq * T + sms >= (1ll << 31)) return cudaErrorInvalidValue;   // the schedule counts items in 32 bits
     if (!lse_in) {
         const long long items = (long long)d.B * d.Hq * T;
         const int grid = (int)(items < sms ? items : sms);
