@@ -103,7 +103,7 @@ int check_ws(const Dims& d, void* ws, size_t ws_bytes, Workspace& w) {
 }
 
 // sim_out (nullable): where the neighbour-key similarities are wanted.  *sim_done tells whether the score
-// step produced them on the side (bf16 row pass) or the caller still has to launch the similarity kernel.
+// step produced them on the side (bf16 path) or the caller still has to launch the similarity kernel.
 cudaError_t run_score(const Dims& d, const void* Q, const void* K, const float* lse_in, float* scores,
                       const Workspace& w, kvm_stats* stats, cudaStream_t st, float* sim_out = nullptr,
                       bool* sim_done = nullptr) {
