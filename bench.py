@@ -44,7 +44,7 @@ N_BUFFERS = 3  # rotating input sets: 3 x 100 MB > 126 MB of L2
 MIN_TIMED_MS = 500.0  # the timed block is repeated until this much GPU time has been measured
 # dram__bytes_read.sum + dram__bytes_write.sum of one column-pass launch on this workload, from the ncu capture
 # summarised in profiles/score_tc_column_pass_C1.md (None when the kernel has changed since that capture)
-NCU_TRAFFIC_BYTES_COLUMN_PASS = 71.42e6 + 3.35e6
+NCU_TRAFFIC_BYTES_COLUMN_PASS = 71.38e6 + 3.14e6
 OTHER_WORKLOADS = ("C2", "C3", "C4")
 LAYERS_PER_WORKLOAD = 3
 
