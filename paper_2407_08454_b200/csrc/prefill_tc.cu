@@ -9,7 +9,11 @@
 // tensor core reads (128-byte rows, 128-byte swizzle) and V read with its head dimension contiguous (the layout
 // it has in memory).  Two groups of four softmax warps take alternate steps, each with its own S accumulator, P
 // tile, O accumulator, reference maximum and row sum, so that one group's exponentials run under the other
-// group's products; the two partial results of a row are joined when the item ends.  A softmax thread owns one
+// group's products; the two partial results of a row are joined when the item ends, by the group that took the
+// item's first step (groups swap from item to item: step j of item n belongs to group (j + n) & 1), which reads
+// the other group's accumulator first and hands it back at once, so that the other group's first step of the next
+// item runs beside the join.  The logits stay two steps ahead of the P V products across item boundaries (the Q
+// tile is released when the item's last Q K^T has been issued).  A softmax thread owns one
 // query row = one TMEM lane: it holds the 128 logits of a step in registers (the accumulator is handed back at
 // once), and multiplies its row of O by exp(old - new reference) only when the maximum has grown by more than
 // 8 (log2 units) since the reference was set, so that most steps touch O not at all.
@@ -48,14 +52,14 @@ struct __align__(8) Bars {
     uint64_t q_full, q_empty;
     uint64_t k_full[NKV], k_empty[NKV], v_full[NKV], v_empty[NKV];
     uint64_t s_full[NGRP], s_empty[NGRP];
-    uint64_t p_full[NGRP], pv_done[NGRP], o_empty;
-    uint64_t part_full, part_empty;     // group 1's row state at item end: written / read
+    uint64_t p_full[NGRP], pv_done[NGRP], o_empty[NGRP];
+    uint64_t part_full, part_empty;     // the handing group's row state at item end: written / read
 };
 struct alignas(16) Shared {
     Bars bar;
     uint32_t tmem_base;
     int abort_flag;
-    float part_m[TILE], part_l[TILE];   // group 1's row state at item end (handed over through part_full / part_empty)
+    float part_m[TILE], part_l[TILE];   // the handing group's row state at item end (through part_full / part_empty)
 };
 
 struct Sched {
@@ -105,7 +109,7 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
             mbar_init(&sh.bar.s_full[i], 1); mbar_init(&sh.bar.s_empty[i], 4);
             mbar_init(&sh.bar.p_full[i], 4); mbar_init(&sh.bar.pv_done[i], 1);
         }
-        mbar_init(&sh.bar.o_empty, 4);
+        for (int i = 0; i < NGRP; ++i) mbar_init(&sh.bar.o_empty[i], 4);
         mbar_init(&sh.bar.part_full, 4); mbar_init(&sh.bar.part_empty, 4);
         sh.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -188,14 +192,35 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                 umma_commit(&sh.bar.s_full[g]);
                 ++ks_cnt; ++s_cnt[g];
             };
+            // Step j of item n belongs to group (j + n) & 1: the group that does not have to join the item's two
+            // partial results starts the next item at once.  The logits run two steps ahead of the P V products,
+            // across item boundaries too: while an item's last products drain, the next item's Q tile is already
+            // on its way (Q is released as soon as the item's last Q K^T has been issued) and its first two S
+            // tiles are computed.
+            int s_n = 0, s_j = 0, s_head, s_tile;            // the next S to issue: item, step
+            bool s_have = sc.item(0, s_head, s_tile);
+            auto advance_s = [&]() {
+                if (!ok || !s_have) return;
+                if (s_j == 0) {
+                    ok = mbar_wait(&sh.bar.q_full, s_n & 1, abort_flag);
+                    if (!ok) return;
+                }
+                issue_s((s_j + s_n) & 1);
+                if (!ok) return;
+                if (s_j == s_tile) {
+                    umma_commit(&sh.bar.q_empty);            // every product that reads this Q tile has been issued
+                    ++s_n; s_j = 0;
+                    s_have = sc.item(s_n, s_head, s_tile);
+                } else {
+                    ++s_j;
+                }
+            };
+            advance_s();
+            advance_s();
             for (int n = 0; ok && sc.item(n, head, tile); ++n) {
-                ok = mbar_wait(&sh.bar.q_full, n & 1, abort_flag);
-                if (!ok) break;
-                issue_s(0);                                  // the logits run two steps ahead of the P V products,
-                if (ok && tile >= 1) issue_s(1);             // one step per group
                 for (int j = 0; ok && j <= tile; ++j) {
-                    const int g = j & 1;
-                    if (j == 0) ok = mbar_wait(&sh.bar.o_empty, (n & 1) ^ 1, abort_flag);   // the last item's O has been read
+                    const int g = (j + n) & 1;
+                    if (j < 2) ok = mbar_wait(&sh.bar.o_empty[g], (n & 1) ^ 1, abort_flag);   // the last item's O of this group has been read
                     const int s = vs_cnt % NKV;
                     ok = ok && mbar_wait(&sh.bar.p_full[g], pv_cnt[g] & 1, abort_flag) &&
                          mbar_wait(&sh.bar.v_full[s], (vs_cnt / NKV) & 1, abort_flag);
@@ -210,9 +235,8 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                     umma_commit(&sh.bar.v_empty[s]);
                     umma_commit(&sh.bar.pv_done[g]);         // the group's P may be overwritten, its O read or rescaled
                     ++vs_cnt; ++pv_cnt[g];
-                    if (j + 2 <= tile) issue_s(g);           // the group has taken its logits into registers long ago
+                    advance_s();
                 }
-                if (ok) umma_commit(&sh.bar.q_empty);
             }
         }
       }
@@ -225,12 +249,13 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
         const uint32_t t_s = t_lane + grp * S_COLS, t_o = t_lane + O_COL0 + grp * S_COLS;
         uint8_t* prow = sP + grp * P_BYTES + row * 128;
         uint32_t s_cnt = 0, pv_cnt = 0;                      // this group's steps so far
-        uint32_t pv_other = 0;                               // the other group's (group 0 reads both results at item end)
+        uint32_t pv_other = 0;                               // the other group's (the joining group reads both results)
         bool ok = true;
         int head, tile;
         for (int n = 0; ok && sc.item(n, head, tile); ++n) {
             float m = -INFINITY, l = 0.f;                    // reference maximum (log2 units) and sum relative to it
-            for (int j = grp; j <= tile; j += NGRP) {
+            const int j_first = (grp + n) & 1;               // this group's first step of the item
+            for (int j = j_first; j <= tile; j += NGRP) {
                 ok = mbar_wait(&sh.bar.s_full[grp], s_cnt & 1, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
@@ -260,7 +285,7 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                 // the reference moves only when the maximum has outgrown it by RESCALE_STEP: exp2(x - m) stays
                 // below 2^RESCALE_STEP, and O is rescaled rarely
                 float alpha = 1.f;
-                const bool first = j == grp;                 // the group's first step of the item
+                const bool first = j == j_first;             // the group's first step of the item
                 const bool grow = mx > m + RESCALE_STEP;
                 if (first) m = mx;
                 else if (grow) { alpha = ex2(m - mx); m = mx; }
@@ -309,13 +334,16 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                 if (lane == 0) mbar_arrive(&sh.bar.p_full[grp]);
                 ++pv_cnt;
             }
-            const int n_other = (tile + 1 + grp) / 2;        // steps the other group takes in this item
+            const int n_own = tile >= j_first ? (tile - j_first) / 2 + 1 : 0;
+            const int n_other = tile + 1 - n_own;            // steps the other group takes in this item
             pv_other += n_other;
-            // ---- item end: group 1 hands its row state to group 0, which joins the two partial results:
-            //      O = (O_0 2^(m_0 - M) + O_1 2^(m_1 - M)) / (l_0 2^(m_0 - M) + l_1 2^(m_1 - M)),  M = max(m_0, m_1)
-            if (grp == 1) {
+            // ---- item end: one group hands its row state to the other, which joins the two partial results:
+            //      O = (O_a 2^(m_a - M) + O_b 2^(m_b - M)) / (l_a 2^(m_a - M) + l_b 2^(m_b - M)),  M = max(m_a, m_b)
+            // The joining group is the one that took the item's first step (group n & 1), so the other one is
+            // free for the next item's first step while the join runs.
+            if (grp != (n & 1)) {
                 // (every item, also one in which this group had no step: the two groups count items alike)
-                ok = ok && mbar_wait(&sh.bar.part_empty, (n & 1) ^ 1, abort_flag);   // group 0 has read the last item's
+                ok = ok && mbar_wait(&sh.bar.part_empty, (n & 1) ^ 1, abort_flag);   // the last item's has been read
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 sh.part_m[row] = m;
@@ -333,8 +361,8 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
             if (ok && lane == 0) mbar_arrive(&sh.bar.part_empty);
             const int gi = tile * TILE + row;
             if (ok) {
-                ok = mbar_wait(&sh.bar.pv_done[0], (pv_cnt & 1) ^ 1, abort_flag);
-                if (ok && n_other > 0) ok = mbar_wait(&sh.bar.pv_done[1], (pv_other & 1) ^ 1, abort_flag);
+                ok = mbar_wait(&sh.bar.pv_done[grp], (pv_cnt & 1) ^ 1, abort_flag);
+                if (ok && n_other > 0) ok = mbar_wait(&sh.bar.pv_done[grp ^ 1], (pv_other & 1) ^ 1, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
             }
             ok = ok && (*abort_flag == 0);
@@ -342,25 +370,38 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
             if (ok) {
                 tc_fence_after();
                 const float M = fmaxf(m, m1);
-                const float w0 = ex2(m - M), w1 = n_other > 0 ? ex2(m1 - M) : 0.f;
+                const float w0 = n_own > 0 ? ex2(m - M) : 0.f, w1 = n_other > 0 ? ex2(m1 - M) : 0.f;
                 const float L = l * w0 + l1 * w1;
                 const float f0 = w0 / L, f1 = w1 / L;
+                // the other group's accumulator first, whole, so that it goes back at once: that group is
+                // already at work on the next item
+                // (a group without a step in this item has a stale accumulator: it is read all the same, so that
+                // the registers are not conditional, and replaced by zeros)
+                uint32_t o1[D];
+#pragma unroll
+                for (int q = 0; q < D / 32; ++q) tmem_ld32_issue(t_lane + O_COL0 + (grp ^ 1) * S_COLS + q * 32, o1 + q * 32);
+                tmem_ld_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh.bar.o_empty[grp ^ 1]);
+#pragma unroll
+                for (int q = 0; q < D / 32; ++q) tmem_ld_fence(o1 + q * 32);
+                const bool has0 = n_own > 0, has1 = n_other > 0;
 #pragma unroll
                 for (int q = 0; q < D / 32; ++q) {
-                    uint32_t o0[32], o1[32];
-                    tmem_ld32_issue(t_lane + O_COL0 + q * 32, o0);
-                    if (n_other > 0) tmem_ld32_issue(t_lane + O_COL0 + S_COLS + q * 32, o1);
+                    uint32_t o0[32];
+                    tmem_ld32_issue(t_o + q * 32, o0);
                     tmem_ld_wait();
                     tmem_ld_fence(o0);
-                    if (n_other > 0) tmem_ld_fence(o1);
                     if (gi < S) {
 #pragma unroll
                         for (int c = 0; c < 32; c += 8) {
                             float f[8];
 #pragma unroll
                             for (int e = 0; e < 8; ++e) {
-                                f[e] = __uint_as_float(o0[c + e]) * f0;
-                                if (n_other > 0) f[e] = fmaf(__uint_as_float(o1[c + e]), f1, f[e]);
+                                const float a0 = has0 ? __uint_as_float(o0[c + e]) : 0.f;
+                                const float a1 = has1 ? __uint_as_float(o1[q * 32 + c + e]) : 0.f;
+                                f[e] = fmaf(a1, f1, a0 * f0);
                             }
                             *reinterpret_cast<uint4*>(orow + q * 32 + c) = Vec<__nv_bfloat16>::pack(f);
                         }
@@ -368,7 +409,7 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&sh.bar.o_empty);
+                if (lane == 0) mbar_arrive(&sh.bar.o_empty[grp]);
                 if (gi < S) lse[(size_t)head * S + gi] = (M + log2f(L)) * LN2;
             } else if (gi < S) {
                 // a wait gave up: what this row would have received is marked, not made up
