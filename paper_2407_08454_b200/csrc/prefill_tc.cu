@@ -19,8 +19,9 @@
 // 8 (log2 units) since the reference was set, so that most steps touch O not at all.
 //
 // One CTA per SM, persistent:  warps 0-7 softmax (group = warp / 4),  warp 8 producer (TMA, 128-byte swizzle; K
-// and V tiles in rings of two),  warp 9 one thread issues the MMAs and owns tensor memory (warps 10-11 only fill the
-// third warpgroup, which gives registers up to the softmax warpgroups).  Items are dealt
+// and V tiles in rings of two),  warp 9 one thread issues the Q K^T MMAs and owns tensor memory,  warp 10 one
+// thread issues the P V MMAs (two issuing threads: neither product's waits hold the other's issue up; warp 11
+// only fills the third warpgroup, which gives registers up to the softmax warpgroups).  Items are dealt
 // longest first, boustrophedon.  Every wait on an mbarrier is bounded; a wait that runs out raises a flag, every
 // role leaves its loops, the rows in hand are written as NaN, kvm_stats.status is set when given, tensor memory
 // is freed.  (The test build of the library, never shipped, shortens the limit and makes the producer leave out one
@@ -164,59 +165,53 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                 for (uint32_t it = 0; it < (1u << 14); ++it) mbar_try(&sh.bar.q_full, 0);
         }
       } else if (warp == NSOFT + 1) {
-        // ============================== MMA issue ==============================
+        // ============================== MMA issue: S = Q K^T ==============================
+        // Step j of item n belongs to group (j + n) & 1.  This thread runs ahead of the P V products as far as the
+        // two S accumulators allow (a group's next S is issued as soon as the group has taken the last one into
+        // registers), across item boundaries too: Q is released as soon as the item's last Q K^T has been issued,
+        // so the next Q tile and the next item's first S tiles arrive while the last products drain.  (Its
+        // commits cover its own MMAs only: the two products are issued by two threads.)
         if (lane == 0) {
-            constexpr uint32_t IDESC_S = idesc_bf16(TILE), IDESC_O = idesc_bf16(D, true);
+            constexpr uint32_t IDESC_S = idesc_bf16(TILE);
             const uint64_t desc_q = smem_desc(base);
             const uint64_t desc_k0 = smem_desc(base + TILE_BYTES);
-            const uint32_t v_addr0 = base + TILE_BYTES + NKV * TILE_BYTES;
-            const uint64_t desc_p0 = smem_desc(v_addr0 + NKV * TILE_BYTES);
-            uint32_t ks_cnt = 0, vs_cnt = 0;                 // K tiles and V tiles consumed so far
-            uint32_t s_cnt[NGRP] = {0, 0}, pv_cnt[NGRP] = {0, 0};   // per group: S tiles produced, P V products issued
+            uint32_t ks_cnt = 0;                             // K tiles consumed so far
+            uint32_t s_cnt[NGRP] = {0, 0};                   // per group: S tiles produced
             bool ok = true;
             int head, tile;
-            auto issue_s = [&](int g) {                      // S of group g = Q K^T with the next K tile
-                const int s = ks_cnt % NKV;
-                ok = mbar_wait(&sh.bar.k_full[s], (ks_cnt / NKV) & 1, abort_flag) &&
-                     mbar_wait(&sh.bar.s_empty[g], (s_cnt[g] & 1) ^ 1, abort_flag);
-                if (!ok) return;
-                tc_fence_after();
-                const uint64_t dk = desc_k0 + (uint64_t)s * (TILE_BYTES >> 4);
+            for (int n = 0; ok && sc.item(n, head, tile); ++n) {
+                ok = mbar_wait(&sh.bar.q_full, n & 1, abort_flag);
+                for (int j = 0; ok && j <= tile; ++j) {
+                    const int g = (j + n) & 1;
+                    const int s = ks_cnt % NKV;
+                    ok = mbar_wait(&sh.bar.k_full[s], (ks_cnt / NKV) & 1, abort_flag) &&
+                         mbar_wait(&sh.bar.s_empty[g], (s_cnt[g] & 1) ^ 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint64_t dk = desc_k0 + (uint64_t)s * (TILE_BYTES >> 4);
 #pragma unroll
-                for (int kc = 0; kc < KCH; ++kc)
+                    for (int kc = 0; kc < KCH; ++kc)
 #pragma unroll
-                    for (int ks = 0; ks < KCHUNK / 16; ++ks)
-                        umma_bf16(tmem_base + g * S_COLS, desc_q + ((kc * CHUNK_BYTES + ks * 32) >> 4),
-                                  dk + ((kc * CHUNK_BYTES + ks * 32) >> 4), IDESC_S, (kc | ks) ? 1u : 0u);
-                umma_commit(&sh.bar.k_empty[s]);
-                umma_commit(&sh.bar.s_full[g]);
-                ++ks_cnt; ++s_cnt[g];
-            };
-            // Step j of item n belongs to group (j + n) & 1: the group that does not have to join the item's two
-            // partial results starts the next item at once.  The logits run two steps ahead of the P V products,
-            // across item boundaries too: while an item's last products drain, the next item's Q tile is already
-            // on its way (Q is released as soon as the item's last Q K^T has been issued) and its first two S
-            // tiles are computed.
-            int s_n = 0, s_j = 0, s_head, s_tile;            // the next S to issue: item, step
-            bool s_have = sc.item(0, s_head, s_tile);
-            auto advance_s = [&]() {
-                if (!ok || !s_have) return;
-                if (s_j == 0) {
-                    ok = mbar_wait(&sh.bar.q_full, s_n & 1, abort_flag);
-                    if (!ok) return;
+                        for (int ks = 0; ks < KCHUNK / 16; ++ks)
+                            umma_bf16(tmem_base + g * S_COLS, desc_q + ((kc * CHUNK_BYTES + ks * 32) >> 4),
+                                      dk + ((kc * CHUNK_BYTES + ks * 32) >> 4), IDESC_S, (kc | ks) ? 1u : 0u);
+                    umma_commit(&sh.bar.k_empty[s]);
+                    umma_commit(&sh.bar.s_full[g]);
+                    ++ks_cnt; ++s_cnt[g];
                 }
-                issue_s((s_j + s_n) & 1);
-                if (!ok) return;
-                if (s_j == s_tile) {
-                    umma_commit(&sh.bar.q_empty);            // every product that reads this Q tile has been issued
-                    ++s_n; s_j = 0;
-                    s_have = sc.item(s_n, s_head, s_tile);
-                } else {
-                    ++s_j;
-                }
-            };
-            advance_s();
-            advance_s();
+                if (ok) umma_commit(&sh.bar.q_empty);        // every product that reads this Q tile has been issued
+            }
+        }
+      } else if (warp == NSOFT + 2) {
+        // ============================== MMA issue: O += P V ==============================
+        if (lane == 0) {
+            constexpr uint32_t IDESC_O = idesc_bf16(D, true);
+            const uint32_t v_addr0 = base + TILE_BYTES + NKV * TILE_BYTES;
+            const uint64_t desc_p0 = smem_desc(v_addr0 + NKV * TILE_BYTES);
+            uint32_t vs_cnt = 0;                             // V tiles consumed so far
+            uint32_t pv_cnt[NGRP] = {0, 0};                  // per group: P V products issued
+            bool ok = true;
+            int head, tile;
             for (int n = 0; ok && sc.item(n, head, tile); ++n) {
                 for (int j = 0; ok && j <= tile; ++j) {
                     const int g = (j + n) & 1;
@@ -226,16 +221,15 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                          mbar_wait(&sh.bar.v_full[s], (vs_cnt / NKV) & 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t va = v_addr0 + s * TILE_BYTES;
+                    const uint64_t dv0 = smem_desc_mn(v_addr0 + s * TILE_BYTES, CHUNK_BYTES);   // 16 keys further: + 2 KB
                     const uint64_t dp = desc_p0 + (uint64_t)g * (P_BYTES >> 4);
 #pragma unroll
                     for (int kk = 0; kk < TILE / 16; ++kk)          // 16 keys per MMA
                         umma_bf16(tmem_base + O_COL0 + g * S_COLS, dp + (((kk / 4) * CHUNK_BYTES + (kk % 4) * 32) >> 4),
-                                  smem_desc_mn(va + kk * 16 * 128, CHUNK_BYTES), IDESC_O, ((j >> 1) | kk) ? 1u : 0u);
+                                  dv0 + (uint64_t)((kk * 16 * 128) >> 4), IDESC_O, ((j >> 1) | kk) ? 1u : 0u);
                     umma_commit(&sh.bar.v_empty[s]);
                     umma_commit(&sh.bar.pv_done[g]);         // the group's P may be overwritten, its O read or rescaled
                     ++vs_cnt; ++pv_cnt[g];
-                    advance_s();
                 }
             }
         }
