@@ -56,6 +56,7 @@ using namespace tc;
 constexpr int TILE = 128;            // rows of an A or B tile = MMA M = MMA N
 constexpr int KCHUNK = 64;           // bf16 elements per 128-byte swizzle row
 constexpr int NSTAGE = 2;            // ring of B pairs (two 128-row tiles each)
+constexpr int NSLOT = 4;             // item-end buffers in rotation
 constexpr int NACC = 2;              // TMEM accumulator ring (2 x 256 columns = all 512)
 constexpr int ACC_COLS = 2 * TILE;   // accumulator columns per step
 constexpr int PCH = 16;              // channels of the lse side tensor (one K = 16 MMA slice; 3 are used)
@@ -166,12 +167,12 @@ struct alignas(16) Shared {
     Barriers bar;
     uint32_t tmem_base;
     int abort_flag;
-    // Row states of the four warp sets at item end, in three buffers used in rotation (item n uses n mod 3:
-    // the warps that share rows are never three items apart, see the item end), and how many of the four
-    // warps that own a lane quarter's rows have delivered theirs.
-    float part_m[3][4][TILE];
-    float part_l[3][4][TILE];
-    int arrived[3][4];
+    // Partial sums of the four warp sets at item end, in NSLOT buffers used in rotation (item n uses n mod
+    // NSLOT; see the item end), and how many of the four warps that own a lane quarter's rows have delivered
+    // theirs.  (The row pass also needs the partial maxima and keeps both arrays where the column pass keeps
+    // its side tiles, which the row pass does not have.)
+    float part_l[NSLOT][4][TILE];
+    int arrived[NSLOT][4];
 };
 
 template <int KCH, int PASS>
@@ -194,6 +195,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     uint8_t* sOnes = sP + NSTAGE * 2 * PTILE_BYTES;         // constant A' tile: ones in the used channels
     Shared& sh = *reinterpret_cast<Shared*>(sOnes + PTILE_BYTES);
     volatile int* abort_flag = &sh.abort_flag;
+    static_assert(2 * NSLOT * 4 * TILE * sizeof(float) <= NSTAGE * 2 * PTILE_BYTES, "the row pass's item-end buffers fit the side tiles' space");
+    float* part_m = reinterpret_cast<float*>(sP);                                   // [NSLOT][4][TILE], row pass only
+    float* part_l = (pass == 1) ? part_m + NSLOT * 4 * TILE : &sh.part_l[0][0][0];     // [NSLOT][4][TILE]
 
     grid_dependency_wait();     // the column pass reads what the row pass (or the lse conversion) wrote
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -206,7 +210,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         for (int i = 0; i < NSTAGE; ++i) { mbar_init(&sh.bar.full_b[i], 1); mbar_init(&sh.bar.empty_b[i], 1); }
         for (int i = 0; i < NACC; ++i) { mbar_init(&sh.bar.acc_full[i], 1); mbar_init(&sh.bar.acc_empty[i], NEPI_WARPS / 2); }
         sh.abort_flag = 0;
-        for (int i = 0; i < 12; ++i) (&sh.arrived[0][0])[i] = 0;
+        for (int i = 0; i < NSLOT * 4; ++i) (&sh.arrived[0][0])[i] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (pass == 2 && threadIdx.x < PTILE_BYTES / 16) {
@@ -441,15 +445,19 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             // state in shared memory; whichever of them comes last combines the four in a fixed order (so the
             // result does not depend on who does it) and stores.  Nobody waits: the group that had the item's
             // last step is a step behind the other one, which goes straight on to the next item.
-            // (Buffers: a warp is at most one step ahead of a warp of the other group, because the MMA thread
-            // needs the slower group's accumulator back before it can issue the step after next; three items
-            // are at least three steps, so the buffer of item n - 3 has been combined when item n's is written.)
-            const int slot = n % 3;
+            // (Buffers: the MMA thread needs a group's accumulator back before it can issue that group's step after
+            // next, and it issues in order; so a warp is at most three steps ahead of a warp of the other group
+            // that has handed its accumulator back but not yet finished its step and its item end.  With
+            // single-step items three steps are three items: four buffers, so that item n - 4 has been
+            // combined, and its count cleared, when item n's states are written.)
+            const int slot = n % NSLOT;
             const float mine = (pass == 1) ? l : ((acc[0] + acc[1]) + (acc[2] + acc[3])) + ((acc[4] + acc[5]) + (acc[6] + acc[7]));
             constexpr int NPART = NEPI_WARPS / 4;            // partial states per row (one per warp that owns it)
             static_assert(NPART == 4, "four warps own a row");
-            sh.part_m[slot][pidx][row] = m;
-            sh.part_l[slot][pidx][row] = mine;
+            float* pm = part_m + slot * 4 * TILE + row;       // + q * TILE: warp set q
+            float* pl = part_l + slot * 4 * TILE + row;
+            if (pass == 1) pm[pidx * TILE] = m;
+            pl[pidx * TILE] = mine;
             __syncwarp();
             int before = 0;
             if (lane == 0) {
@@ -459,20 +467,20 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             before = __shfl_sync(0xffffffffu, before, 0);
             if (before == NPART - 1) {
                 __threadfence_block();
-                if (lane == 0) sh.arrived[slot][lq] = 0;     // for item n + 3
+                if (lane == 0) sh.arrived[slot][lq] = 0;     // for item n + NSLOT
                 // (read after all four have delivered: a warp whose wait ran out raised the flag before it came here)
                 const bool bad = (*abort_flag != 0);
                 const int gi = tile * TILE + row;
                 if (gi < S) {
                     if (pass == 1) {
-                        const float m0 = sh.part_m[slot][0][row];
+                        const float m0 = pm[0];
                         float M = m0;
 #pragma unroll
-                        for (int q = 1; q < NPART; ++q) M = fmaxf(M, sh.part_m[slot][q][row]);
-                        float L = (m0 > -INFINITY) ? sh.part_l[slot][0][row] * ex2(m0 - M) : 0.f;
+                        for (int q = 1; q < NPART; ++q) M = fmaxf(M, pm[q * TILE]);
+                        float L = (m0 > -INFINITY) ? pl[0] * ex2(m0 - M) : 0.f;
 #pragma unroll
                         for (int q = 1; q < NPART; ++q) {
-                            const float mq = sh.part_m[slot][q][row], lq_ = sh.part_l[slot][q][row];
+                            const float mq = pm[q * TILE], lq_ = pl[q * TILE];
                             if (mq > -INFINITY) L += lq_ * ex2(mq - M);
                         }
                         // e = -lse / c in the accumulator's units (lse in log2 units is M + log2 L), as hi + mid + lo
@@ -486,9 +494,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                                             (uint32_t)__bfloat16_as_ushort(el), 0u, 0u);
                         dst[1] = make_uint4(0u, 0u, 0u, 0u);
                     } else {
-                        float tot = sh.part_l[slot][0][row];
+                        float tot = pl[0];
 #pragma unroll
-                        for (int q = 1; q < NPART; ++q) tot += sh.part_l[slot][q][row];
+                        for (int q = 1; q < NPART; ++q) tot += pl[q * TILE];
                         scores[(size_t)head * S + gi] = bad ? NAN : tot / (float)G;
                     }
                 }

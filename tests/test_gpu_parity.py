@@ -74,6 +74,19 @@ def test_budget_rule_fires_on_a_sequence_beyond_the_register_kernel():
     check_case(case)
 
 
+def test_many_single_step_work_items_per_cta():
+    """Short sequences and many heads: every work item of the score passes is a single step, a CTA runs through
+    several of them in a row, and the warps that share a row's partial state run items apart from one another
+    (the rotating item-end buffers and their use counts).  Against the checker, and twice for identical bits."""
+    cfg = si.CONFIGS["C1"].scaled(seq=256, n_q_heads=64, n_kv_heads=64, batch=8, seed=31)
+    case = _case(cfg)
+    g1 = run_gpu(case)
+    check_case(case, g1)
+    for _ in range(3):
+        g2 = run_gpu(case)
+        assert np.array_equal(g1.c_scores, g2.c_scores) and np.array_equal(g1.c_K_out, g2.c_K_out)
+
+
 def test_threshold_above_one_returns_the_input_cache():
     cfg = si.CONFIGS["C1"].scaled(seq=512, n_q_heads=2, n_kv_heads=2, seed=8)
     d = si.make_layer(cfg)
