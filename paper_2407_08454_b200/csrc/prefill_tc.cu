@@ -18,10 +18,10 @@
 // once), and multiplies its row of O by exp(old - new reference) only when the maximum has grown by more than
 // 8 (log2 units) since the reference was set, so that most steps touch O not at all.
 //
-// One CTA per SM, persistent:  warps 0-7 softmax (group = warp / 4),  warp 8 producer (TMA, 128-byte swizzle; K
-// and V tiles in rings of two),  warp 9 one thread issues the Q K^T MMAs and owns tensor memory,  warp 10 one
-// thread issues the P V MMAs (two issuing threads: neither product's waits hold the other's issue up; warp 11
-// only fills the third warpgroup, which gives registers up to the softmax warpgroups).  Items are dealt
+// One CTA per SM, persistent:  warps 0-7 softmax (group = warp / 4),  warp 8 producer of the Q and K tiles (TMA,
+// 128-byte swizzle; K and V tiles in rings of two),  warp 9 one thread issues the Q K^T MMAs and owns tensor memory,  warp 10 one
+// thread issues the P V MMAs (two issuing threads: neither product's waits hold the other's issue up),  warp 11
+// producer of the V tiles (the third warpgroup gives registers up to the softmax warpgroups).  Items are dealt
 // longest first, boustrophedon.  Every wait on an mbarrier is bounded; a wait that runs out raises a flag, every
 // role leaves its loops, the rows in hand are written as NaN, kvm_stats.status is set when given, tensor memory
 // is freed.  (The test build of the library, never shipped, shortens the limit and makes the producer leave out one
@@ -124,9 +124,11 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
     if (warp >= NSOFT) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_OTHER));
       if (warp == NSOFT) {
-        // ============================== producer ==============================
+        // ============================== producer of the Q and K tiles ==============================
+        // (The V tiles have a producer of their own: a V tile's slot comes free a step or two after the K tile's
+        // of the same step, and one thread loading both in turn would hold the next K tile back behind that wait.)
         if (lane == 0) {
-            uint32_t kv = 0;                                  // K/V tiles loaded so far
+            uint32_t kv = 0;                                  // K tiles loaded so far
             bool ok = true;
             int head, tile;
             for (int n = 0; ok && sc.item(n, head, tile); ++n) {
@@ -139,18 +141,34 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                 const int kvhead = (head / Hq) * Hkv + (head % Hq) / G;
                 for (int j = 0; j <= tile; ++j, ++kv) {
                     const int s = kv % NKV;
-                    const uint32_t par = ((kv / NKV) & 1) ^ 1;
-                    ok = mbar_wait(&sh.bar.k_empty[s], par, abort_flag);
+                    ok = mbar_wait(&sh.bar.k_empty[s], ((kv / NKV) & 1) ^ 1, abort_flag);
                     if (!ok) break;
                     mbar_expect_tx(&sh.bar.k_full[s], TILE_BYTES);
 #pragma unroll
                     for (int kc = 0; kc < KCH; ++kc)
                         tma_load_3d(sK + s * TILE_BYTES + kc * CHUNK_BYTES, &map_k, &sh.bar.k_full[s], kc * KCHUNK,
                                     j * TILE, kvhead);
+                }
+            }
+            // Copies already issued complete on their own; before shared memory is given back, let them land
+            // (bounded: each try_wait suspends for a while by itself).
+            if (*abort_flag)
+                for (uint32_t it = 0; it < (1u << 14); ++it) mbar_try(&sh.bar.q_full, 0);
+        }
+      } else if (warp == NSOFT + 3) {
+        // ============================== producer of the V tiles ==============================
+        if (lane == 0) {
+            uint32_t kv = 0;                                  // V tiles loaded so far
+            bool ok = true;
+            int head, tile;
+            for (int n = 0; ok && sc.item(n, head, tile); ++n) {
+                const int kvhead = (head / Hq) * Hkv + (head % Hq) / G;
+                for (int j = 0; j <= tile; ++j, ++kv) {
 #ifdef KVM_TEST_DROP_B_STAGE
                     if (kv == (uint32_t)(KVM_TEST_DROP_B_STAGE)) continue;   // test build only: this V tile never arrives
 #endif
-                    ok = mbar_wait(&sh.bar.v_empty[s], par, abort_flag);
+                    const int s = kv % NKV;
+                    ok = mbar_wait(&sh.bar.v_empty[s], ((kv / NKV) & 1) ^ 1, abort_flag);
                     if (!ok) break;
                     mbar_expect_tx(&sh.bar.v_full[s], TILE_BYTES);
 #pragma unroll
@@ -159,10 +177,8 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                                     j * TILE, kvhead);
                 }
             }
-            // Copies already issued complete on their own; before shared memory is given back, let them land
-            // (bounded: each try_wait suspends for a while by itself).
             if (*abort_flag)
-                for (uint32_t it = 0; it < (1u << 14); ++it) mbar_try(&sh.bar.q_full, 0);
+                for (uint32_t it = 0; it < (1u << 14); ++it) mbar_try(&sh.bar.v_full[0], 0);
         }
       } else if (warp == NSOFT + 1) {
         // ============================== MMA issue: S = Q K^T ==============================
